@@ -1,0 +1,243 @@
+/*
+ * psd.h — C ABI of the PSD (Parallel Speculative Decoding for diffusion LLMs) per-step hot path
+ * for NVIDIA B200 (sm_100a).
+ *
+ * One decoding step of PSD, seen from the LM head onwards, is four operations:
+ *
+ *   psd_confidence      x^_i = argmax_v p(v), c_i = max_v p(v) for every row of final hidden
+ *                       states, p = softmax(hidden · W_lm^T)            (Sec. 3.1; Sec. 3.2 Stage 3)
+ *   psd_verify_accept   hierarchical acceptance of a chain of drafts    (Sec. 3.2 Stage 3; Alg. 1 Stage 3)
+ *   psd_select_unmask   transfer policy pi and the state update          (Sec. 3.2 Stage 1; Eq. (1))
+ *   psd_build_drafts    speculative ordering sigma and draft assembly    (Sec. 3.2 Stage 2; Eq. (2))
+ *
+ * Conventions, common to every entry point unless it says otherwise:
+ *   - Every array pointer is a DEVICE pointer owned by the caller.  The library allocates no
+ *     device memory and keeps no state between calls.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream).  Outputs are valid once the stream has reached the end of the call.
+ *   - The return value is PSD_OK or a negative psd_status code.  Argument errors are detected
+ *     on the host before anything is launched; nothing is written in that case.
+ *   - Layouts are row-major and dense.  A "block" is one sequence's active block of M slots.
+ *     B = blocks, D = chain nodes per block in the verification batch (root included; the paper's
+ *     draft depth d equals D-1), rows of the verification batch are ordered (b, d, i):
+ *     row = (b*D + d)*M + i.
+ *   - mask arrays hold 1 for a masked slot ([M] in the paper) and 0 for a committed one.
+ *   - No exceptions, no output on stdout/stderr, plain C linkage.
+ */
+#ifndef PSD_H_
+#define PSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum psd_status {
+    PSD_OK = 0,
+    PSD_ERR_NULL = -1,        /* a required pointer is NULL                                        */
+    PSD_ERR_SHAPE = -2,       /* a size is out of range (see each call)                            */
+    PSD_ERR_ALIGN = -3,       /* a pointer is not aligned as required                              */
+    PSD_ERR_WORKSPACE = -4,   /* workspace smaller than psd_workspace_bytes()                      */
+    PSD_ERR_POLICY = -5,      /* k_min < 1, 0 < k_max < k_min, depth out of range, stride < 0,
+                                 unknown accept_mode, or tau is NaN                                 */
+    PSD_ERR_CUDA = -6,        /* a CUDA runtime or driver call failed (launch, tensor-map encode)  */
+    PSD_ERR_UNSUPPORTED = -7, /* a reserved argument was used                                      */
+    PSD_ERR_TIMEOUT = -8      /* device side only, via status_dev: a bounded wait inside a kernel
+                                 ran out; the kernel returned early and its outputs are invalid    */
+} psd_status;
+
+/* Limits checked by the entry points. */
+#define PSD_MAX_M 1024     /* slots per block                        */
+#define PSD_MAX_DEPTH 64   /* chain nodes per block, root included   */
+
+/* accept_mode: the form of the acceptance criterion A_pi(x~_{k,i}, x^_{p,i}, c_{p,i}) of
+ * Algorithm 1 (the paper gives "sufficient confidence" as its example and leaves the form open). */
+#define PSD_ACCEPT_AGREE_AND_CONF 0   /* x~ == x^_p  and  c_p > tau              (default) */
+#define PSD_ACCEPT_AGREE_ONLY 1       /* x~ == x^_p                                         */
+#define PSD_ACCEPT_AGREE_AND_POLICY 2 /* x~ == x^_p  and  i is in pi(parent's draft, c_p)  */
+
+/*
+ * Parameters of the transfer policy and of the draft chain, passed by value.
+ *
+ * The policy is confidence thresholding (App. B.2: unmask every masked position whose top-1
+ * confidence exceeds tau, strictly), clamped to at least k_min positions (so that the decoding
+ * loop of Algorithm 1 always progresses) and at most k_max.  k_min = k_max = 1 is greedy decoding,
+ * k_min = k_max = k is fixed-k parallel decoding (Sec. 2.1).
+ */
+typedef struct psd_policy_t {
+    float tau;           /* commit / acceptance threshold, compared with '>' in fp32              */
+    int32_t k_min;       /* >= 1                                                                  */
+    int32_t k_max;       /* >= k_min, or 0 for "no cap"                                           */
+    int32_t depth;       /* D, 1 .. PSD_MAX_DEPTH; D = 1 means no speculation                     */
+    int32_t stride;      /* slots each further depth speculates; 0 means k_min                    */
+    int32_t accept_mode; /* PSD_ACCEPT_*                                                          */
+    int32_t mask_id;     /* token id of [M]; written to no output, kept for callers' bookkeeping  */
+} psd_policy_t;
+
+/* Text for a psd_status code (static storage, never NULL). */
+const char* psd_status_string(int code);
+
+/*
+ * Bytes of scratch that psd_confidence needs for n_rows x H x V.  Returns 0 for invalid sizes.
+ * The scratch holds the per-row partial (max, sum-exp, argmax) triples of every vocabulary split.
+ */
+size_t psd_workspace_bytes(int32_t n_rows, int32_t H, int32_t V);
+
+/*
+ * psd_confidence — LM head + softmax max-probability + argmax, without ever storing logits.
+ * (Sec. 3.1: x^_i and c_i; used for the single sequence of Stage 1 and for all drafts of the
+ *  batched verification pass of Stage 3.)
+ *
+ * For each row r:  l_v = sum_j hidden[r,j] * w_lm[v,j]  (bf16 inputs, fp32 accumulation),
+ *   out_token[r] = the lowest v attaining max_v l_v,
+ *   out_conf[r]  = 1 / sum_v exp(l_v - max_v l_v)   ( = max_v softmax(l)_v ),
+ *   out_lse[r]   = max_v l_v + ln sum_v exp(l_v - max_v l_v)      (optional).
+ *
+ *   hidden_bf16  [n_rows, H] bf16, 16-byte aligned, device
+ *   w_lm_bf16    [V, H]      bf16, 16-byte aligned, device
+ *   row_ids      reserved for a gather list of active rows; must be NULL
+ *   n_rows >= 1;  H >= 64 and a multiple of 64;  1 <= V < 2^31 - 256
+ *   out_token    [n_rows] int32;  out_conf [n_rows] fp32;  out_lse [n_rows] fp32 or NULL
+ *   workspace    >= psd_workspace_bytes(n_rows, H, V) bytes, 256-byte aligned, device; contents
+ *                are overwritten; concurrent calls need distinct workspaces
+ *   status_dev   NULL, or a device int32 that the caller zeroed: receives PSD_ERR_TIMEOUT if a
+ *                bounded wait inside the kernel expired (outputs are then invalid)
+ * Rows whose logits contain NaN produce out_conf = NaN.
+ */
+int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_ids,
+                   int32_t n_rows, int32_t H, int32_t V,
+                   int32_t* out_token, float* out_conf, float* out_lse,
+                   void* workspace, size_t workspace_bytes,
+                   int32_t* status_dev, void* cuda_stream);
+
+/*
+ * psd_select_unmask — the transfer policy T = pi(x, c) and the state update of Eq. (1).
+ * (Sec. 3.2 Stage 1; App. B.2 for the threshold rule.)
+ *
+ * conf, tok are [B, n_nodes, M]; block b reads the rows of node node[b] (node 0 when node is
+ * NULL).  Over the masked slots of block b, ranked by (confidence descending, slot ascending; NaN
+ * last):  n_thr = #{c_i > tau},  n = min(#masked, k_max or inf, max(n_thr, k_min)),  T = the first
+ * n.  Then tokens[b,i] = tok[i] and mask[b,i] = 0 for i in T; every other slot is left untouched.
+ *
+ *   tokens, mask [B, M] int32, in/out
+ *   sel      [B, M] int32 out: 1 where i in T, else 0
+ *   n_sel    [B]    int32 out: |T|
+ *   sel_pos  [B, M] int32 out: the slots of T in rank order, then -1
+ *   1 <= B; 1 <= M <= PSD_MAX_M; 1 <= n_nodes <= PSD_MAX_DEPTH; node values must lie in [0, n_nodes)
+ */
+int psd_select_unmask(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
+                      int32_t* tokens, int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
+                      int32_t* sel, int32_t* n_sel, int32_t* sel_pos, void* cuda_stream);
+
+/*
+ * psd_build_drafts — speculative ordering and draft assembly for a chain of D = p.depth nodes.
+ * (Sec. 3.2 Stage 2; Eq. (2); Algorithm 1 Stage 2.)
+ *
+ * conf, tok [B, n_nodes, M] are the cached predictions the step started from (node selection as in
+ * psd_select_unmask); tokens, mask [B, M] are the state AFTER psd_select_unmask.  With m masked
+ * slots left, sigma orders them by (cached confidence descending, slot ascending; NaN last);
+ * node d fills S_d = {sigma_1 .. sigma_{n_d}}, n_d = min(m, d * s), s = stride or k_min:
+ *   draft_tokens[b,d,i] = tok[i] if i in S_d else tokens[b,i];   draft_mask[b,d,i] = mask[b,i] and i not in S_d.
+ * Node 0 is the root (S_0 empty).  A block with m = 0 yields D copies of its state and n_fill = 0.
+ *
+ *   sigma   [B, M] int32 out, -1 after the first m entries
+ *   n_fill  [B, D] int32 out
+ *   draft_tokens, draft_mask [B, D, M] int32 out
+ */
+int psd_build_drafts(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
+                     const int32_t* tokens, const int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
+                     int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens, int32_t* draft_mask,
+                     void* cuda_stream);
+
+/*
+ * psd_verify_accept — hierarchical acceptance over the chain, then the commit.
+ * (Sec. 3.2 Stage 3; Algorithm 1 Stage 3.)
+ *
+ * tokV, confV [B, D, M] are psd_confidence's outputs on the D drafts built by psd_build_drafts
+ * (sigma, n_fill, draft_tokens, draft_mask as written there, D = p.depth).  Node 0 is accepted;
+ * node d >= 1 is accepted iff node d-1 is and every slot i = sigma_j, n_{d-1} < j <= n_d, passes
+ * A_pi against node d-1's predictions (p.accept_mode).  k* is the accepted node that fills the
+ * most slots, lowest index among equals.  Then tokens, mask <- draft k*, and every slot still
+ * masked in draft k* whose confV[b,k*,i] > tau is committed to tokV[b,k*,i] as well.
+ *
+ *   tokens, mask     [B, M] int32 out (fully written)
+ *   k_star           [B] int32 out
+ *   n_spec_accepted  [B] int32 out: n_fill[b, k*]
+ *   n_committed      [B] int32 out: n_spec_accepted plus the extra commits
+ *   accepted         [B, D] int32 out or NULL: 1 for accepted nodes
+ */
+int psd_verify_accept(const int32_t* tokV, const float* confV,
+                      const int32_t* sigma, const int32_t* n_fill,
+                      const int32_t* draft_tokens, const int32_t* draft_mask,
+                      int32_t B, int32_t M, psd_policy_t p,
+                      int32_t* tokens, int32_t* mask,
+                      int32_t* k_star, int32_t* n_spec_accepted, int32_t* n_committed,
+                      int32_t* accepted, void* cuda_stream);
+
+/*
+ * All pointers of one decoding step over a batch of B blocks.  Device pointers for psd_step,
+ * HOST pointers (pinned memory recommended) for psd_step_host, except w_lm_bf16 which is a
+ * device pointer in both.
+ */
+typedef struct psd_step_io_t {
+    const void* hidden_bf16;  /* in  [B*D*M, H] final hidden states of the verification batch      */
+    const void* w_lm_bf16;    /* in  [V, H] DEVICE                                                 */
+    int32_t* sigma;           /* in/out [B, M]    drafts being verified -> drafts for the next step */
+    int32_t* n_fill;          /* in/out [B, D]                                                     */
+    int32_t* draft_tokens;    /* in/out [B, D, M]                                                  */
+    int32_t* draft_mask;      /* in/out [B, D, M]                                                  */
+    int32_t* tokV;            /* out [B, D, M] verifier predictions                                */
+    float* confV;             /* out [B, D, M] verifier confidences                                */
+    int32_t* tokens;          /* out [B, M] state after acceptance and the policy                  */
+    int32_t* mask;            /* out [B, M]                                                        */
+    int32_t* k_star;          /* out [B]                                                           */
+    int32_t* n_spec_accepted; /* out [B]                                                           */
+    int32_t* n_committed;     /* out [B] acceptance commits (the policy's are in n_sel)            */
+    int32_t* sel;             /* out [B, M]                                                        */
+    int32_t* n_sel;           /* out [B]                                                           */
+    int32_t* sel_pos;         /* out [B, M]                                                        */
+} psd_step_io_t;
+
+/*
+ * psd_step — one whole step on device buffers, on one stream, with no host synchronisation:
+ *   psd_confidence on all B*D*M rows  ->  psd_verify_accept on the drafts in io
+ *   ->  psd_select_unmask on node k*'s predictions  ->  psd_build_drafts for the next step
+ * (the verification pass of Algorithm 1 doubles as the model call of the next iteration).
+ * Argument rules are those of the four calls; D = p.depth.
+ */
+int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+             void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
+ * Bytes of device staging that psd_step_host needs (inputs, outputs and psd_confidence's
+ * scratch).  Returns 0 for invalid sizes.
+ */
+size_t psd_step_host_bytes(int32_t B, int32_t M, int32_t H, int32_t V, int32_t D);
+
+/*
+ * psd_step_host — psd_step for callers whose per-step data lives in host memory.
+ * Copies hidden and the draft state host->device into `staging`, runs psd_step, copies every
+ * output of io back device->host, and waits for the stream.  io holds HOST pointers
+ * (w_lm_bf16 excepted).  staging: device, 256-byte aligned, >= psd_step_host_bytes().
+ * status_host: NULL, or receives the device status word (PSD_OK or PSD_ERR_TIMEOUT).
+ * Synchronous: returns after the outputs are in host memory.
+ */
+int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+                  void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream);
+
+/*
+ * Which kernel psd_confidence uses: 0 = the tcgen05/TMA kernel (default), 1 = a plain
+ * CUDA-core kernel kept for cross-checking.  Process-wide; returns the previous value, or
+ * PSD_ERR_SHAPE for an unknown value.
+ */
+int psd_set_confidence_impl(int impl);
+
+/* Number of kernel launches the library has issued in this process (all entry points). */
+int64_t psd_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSD_H_ */

@@ -1,0 +1,223 @@
+"""ctypes binding of libpsd_b200.so: the same entry points as include/psd.h, argument marshalling only.
+
+Tensor arguments are torch tensors (device tensors for the device entry points, pinned or plain
+host tensors for ``psd_step_host``); every step of the path runs inside the library's CUDA
+kernels.  There is no fallback: if the shared library cannot be loaded the import of this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+_i32, _i64, _f32, _vp, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+
+PSD_OK = 0
+PSD_ERR_NULL, PSD_ERR_SHAPE, PSD_ERR_ALIGN, PSD_ERR_WORKSPACE = -1, -2, -3, -4
+PSD_ERR_POLICY, PSD_ERR_CUDA, PSD_ERR_UNSUPPORTED, PSD_ERR_TIMEOUT = -5, -6, -7, -8
+PSD_MAX_M, PSD_MAX_DEPTH = 1024, 64
+ACCEPT_AGREE_AND_CONF, ACCEPT_AGREE_ONLY, ACCEPT_AGREE_AND_POLICY = 0, 1, 2
+
+
+class PsdPolicy(ctypes.Structure):
+    """psd_policy_t"""
+    _fields_ = [("tau", _f32), ("k_min", _i32), ("k_max", _i32), ("depth", _i32), ("stride", _i32),
+                ("accept_mode", _i32), ("mask_id", _i32)]
+
+
+class PsdStepIO(ctypes.Structure):
+    """psd_step_io_t"""
+    _fields_ = [(n, _vp) for n in ("hidden_bf16", "w_lm_bf16", "sigma", "n_fill", "draft_tokens", "draft_mask",
+                                   "tokV", "confV", "tokens", "mask", "k_star", "n_spec_accepted",
+                                   "n_committed", "sel", "n_sel", "sel_pos")]
+
+
+class PsdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    lib = ctypes.CDLL(path)
+    pol = PsdPolicy
+    lib.psd_status_string.restype = ctypes.c_char_p
+    lib.psd_status_string.argtypes = [ctypes.c_int]
+    lib.psd_workspace_bytes.restype = _sz
+    lib.psd_workspace_bytes.argtypes = [_i32, _i32, _i32]
+    lib.psd_confidence.restype = ctypes.c_int
+    lib.psd_confidence.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    lib.psd_select_unmask.restype = ctypes.c_int
+    lib.psd_select_unmask.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, pol, _vp, _vp, _vp, _vp]
+    lib.psd_build_drafts.restype = ctypes.c_int
+    lib.psd_build_drafts.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, pol, _vp, _vp, _vp, _vp, _vp]
+    lib.psd_verify_accept.restype = ctypes.c_int
+    lib.psd_verify_accept.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, pol, _vp, _vp, _vp, _vp, _vp,
+                                      _vp, _vp]
+    lib.psd_step.restype = ctypes.c_int
+    lib.psd_step.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
+    lib.psd_step_host_bytes.restype = _sz
+    lib.psd_step_host_bytes.argtypes = [_i32, _i32, _i32, _i32, _i32]
+    lib.psd_step_host.restype = ctypes.c_int
+    lib.psd_step_host.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
+    lib.psd_set_confidence_impl.restype = ctypes.c_int
+    lib.psd_set_confidence_impl.argtypes = [ctypes.c_int]
+    lib.psd_launch_count.restype = _i64
+    lib.psd_launch_count.argtypes = []
+    return lib
+
+
+LIB = _load()
+LIB_PATH = _build.LIB
+
+
+def status_string(code: int) -> str:
+    return LIB.psd_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != PSD_OK:
+        raise PsdError(code, where)
+
+
+def _ptr(t):
+    """Address of a tensor's first element, or None."""
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("psd binding: tensors must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def policy(tau=0.9, k_min=1, k_max=0, depth=1, stride=0, accept_mode=0, mask_id=0) -> PsdPolicy:
+    return PsdPolicy(float(tau), int(k_min), int(k_max), int(depth), int(stride), int(accept_mode), int(mask_id))
+
+
+def psd_workspace_bytes(n_rows: int, H: int, V: int) -> int:
+    return int(LIB.psd_workspace_bytes(n_rows, H, V))
+
+
+def psd_set_confidence_impl(impl: int) -> int:
+    return int(LIB.psd_set_confidence_impl(int(impl)))
+
+
+def psd_launch_count() -> int:
+    return int(LIB.psd_launch_count())
+
+
+def psd_confidence(hidden, w_lm, out_token, out_conf, out_lse=None, workspace=None, status=None, stream=None,
+                   row_ids=None):
+    """hidden [n_rows, H] bf16, w_lm [V, H] bf16 -> out_token int32, out_conf fp32 (and out_lse) [n_rows]."""
+    n_rows, H = hidden.shape
+    V = w_lm.shape[0]
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(LIB.psd_confidence(_ptr(hidden), _ptr(w_lm), _ptr(row_ids), n_rows, H, V, _ptr(out_token),
+                              _ptr(out_conf), _ptr(out_lse), _ptr(workspace), ws_bytes, _ptr(status),
+                              _stream(stream)), "psd_confidence")
+
+
+def psd_select_unmask(conf, tok, tokens, mask, p: PsdPolicy, sel, n_sel, sel_pos, node=None, n_nodes=1,
+                      stream=None):
+    B, M = mask.shape
+    _check(LIB.psd_select_unmask(_ptr(conf), _ptr(tok), _ptr(node), n_nodes, _ptr(tokens), _ptr(mask), B, M, p,
+                                 _ptr(sel), _ptr(n_sel), _ptr(sel_pos), _stream(stream)), "psd_select_unmask")
+
+
+def psd_build_drafts(conf, tok, tokens, mask, p: PsdPolicy, sigma, n_fill, draft_tokens, draft_mask, node=None,
+                     n_nodes=1, stream=None):
+    B, M = mask.shape
+    _check(LIB.psd_build_drafts(_ptr(conf), _ptr(tok), _ptr(node), n_nodes, _ptr(tokens), _ptr(mask), B, M, p,
+                                _ptr(sigma), _ptr(n_fill), _ptr(draft_tokens), _ptr(draft_mask), _stream(stream)),
+           "psd_build_drafts")
+
+
+def psd_verify_accept(tokV, confV, sigma, n_fill, draft_tokens, draft_mask, p: PsdPolicy, tokens, mask, k_star,
+                      n_spec_accepted, n_committed, accepted=None, stream=None):
+    B, M = tokens.shape
+    _check(LIB.psd_verify_accept(_ptr(tokV), _ptr(confV), _ptr(sigma), _ptr(n_fill), _ptr(draft_tokens),
+                                 _ptr(draft_mask), B, M, p, _ptr(tokens), _ptr(mask), _ptr(k_star),
+                                 _ptr(n_spec_accepted), _ptr(n_committed), _ptr(accepted), _stream(stream)),
+           "psd_verify_accept")
+
+
+_STEP_FIELDS = [n for n, _ in PsdStepIO._fields_]
+
+
+@dataclass
+class StepBuffers:
+    """The tensors of one decoding step (psd_step_io_t), all on one device or all on the host
+    (``w_lm`` always on the device)."""
+    hidden: torch.Tensor
+    w_lm: torch.Tensor
+    sigma: torch.Tensor
+    n_fill: torch.Tensor
+    draft_tokens: torch.Tensor
+    draft_mask: torch.Tensor
+    tokV: torch.Tensor
+    confV: torch.Tensor
+    tokens: torch.Tensor
+    mask: torch.Tensor
+    k_star: torch.Tensor
+    n_spec_accepted: torch.Tensor
+    n_committed: torch.Tensor
+    sel: torch.Tensor
+    n_sel: torch.Tensor
+    sel_pos: torch.Tensor
+
+    def io(self) -> PsdStepIO:
+        vals = [self.hidden, self.w_lm, self.sigma, self.n_fill, self.draft_tokens, self.draft_mask, self.tokV,
+                self.confV, self.tokens, self.mask, self.k_star, self.n_spec_accepted, self.n_committed, self.sel,
+                self.n_sel, self.sel_pos]
+        return PsdStepIO(*[_ptr(v) for v in vals])
+
+    @staticmethod
+    def allocate(B, M, D, H, hidden, w_lm, device, pin=False):
+        kw = dict(device=device)
+        if pin:
+            kw["pin_memory"] = True
+        i32 = lambda *s: torch.zeros(*s, dtype=torch.int32, **kw)
+        return StepBuffers(hidden=hidden, w_lm=w_lm, sigma=i32(B, M), n_fill=i32(B, D), draft_tokens=i32(B, D, M),
+                           draft_mask=i32(B, D, M), tokV=i32(B, D, M),
+                           confV=torch.zeros(B, D, M, dtype=torch.float32, **kw), tokens=i32(B, M), mask=i32(B, M),
+                           k_star=i32(B), n_spec_accepted=i32(B), n_committed=i32(B), sel=i32(B, M), n_sel=i32(B),
+                           sel_pos=i32(B, M))
+
+
+def psd_step(buf: StepBuffers, p: PsdPolicy, workspace, status=None, stream=None):
+    B, M = buf.tokens.shape
+    H = buf.hidden.shape[1]
+    V = buf.w_lm.shape[0]
+    io = buf.io()
+    _check(LIB.psd_step(ctypes.byref(io), B, M, H, V, p, _ptr(workspace),
+                        workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)), "psd_step")
+
+
+def psd_step_host_bytes(B, M, H, V, D) -> int:
+    return int(LIB.psd_step_host_bytes(B, M, H, V, D))
+
+
+def psd_step_host(buf: StepBuffers, p: PsdPolicy, staging, stream=None) -> int:
+    """``buf`` holds host tensors (w_lm on the device).  Returns the device status word."""
+    B, M = buf.tokens.shape
+    H = buf.hidden.shape[1]
+    V = buf.w_lm.shape[0]
+    io = buf.io()
+    st = _i32(0)
+    _check(LIB.psd_step_host(ctypes.byref(io), B, M, H, V, p, _ptr(staging),
+                             staging.numel() * staging.element_size(), ctypes.byref(st), _stream(stream)),
+           "psd_step_host")
+    return int(st.value)

@@ -1,0 +1,260 @@
+// extern "C" entry points of libpsd_b200: argument checking, then kernel launches.  See psd.h.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include "psd_internal.cuh"
+
+namespace psd {
+namespace {
+std::atomic<long long> g_launches{0};
+std::atomic<int> g_conf_impl{0};
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_policy(const psd_policy_t& p) {
+    if (p.k_min < 1 || (p.k_max != 0 && p.k_max < p.k_min) || p.depth < 1 || p.depth > PSD_MAX_DEPTH ||
+        p.stride < 0 || p.accept_mode < 0 || p.accept_mode > 2 || std::isnan(p.tau))
+        return PSD_ERR_POLICY;
+    return PSD_OK;
+}
+
+int check_block_shape(int B, int M) { return (B < 1 || M < 1 || M > PSD_MAX_M) ? PSD_ERR_SHAPE : PSD_OK; }
+
+bool conf_shape_ok(int n_rows, int H, int V) {
+    return n_rows >= 1 && H >= 64 && H % 64 == 0 && V >= 1 && V < 2147483647 - 256;
+}
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace psd
+
+using namespace psd;
+
+extern "C" {
+
+const char* psd_status_string(int code) {
+    switch (code) {
+        case PSD_OK: return "ok";
+        case PSD_ERR_NULL: return "a required pointer is NULL";
+        case PSD_ERR_SHAPE: return "a size is out of range";
+        case PSD_ERR_ALIGN: return "a pointer is not sufficiently aligned";
+        case PSD_ERR_WORKSPACE: return "workspace too small";
+        case PSD_ERR_POLICY: return "invalid policy parameters";
+        case PSD_ERR_CUDA: return "a CUDA call failed";
+        case PSD_ERR_UNSUPPORTED: return "a reserved argument was used";
+        case PSD_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+        default: return "unknown status";
+    }
+}
+
+size_t psd_workspace_bytes(int32_t n_rows, int32_t H, int32_t V) {
+    if (!conf_shape_ok(n_rows, H, V)) return 0;
+    return round_up((size_t)max_splits(V) * (size_t)n_rows * 12, 256);
+}
+
+int psd_set_confidence_impl(int impl) {
+    if (impl != 0 && impl != 1) return PSD_ERR_SHAPE;
+    return g_conf_impl.exchange(impl);
+}
+
+int64_t psd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_ids,
+                   int32_t n_rows, int32_t H, int32_t V,
+                   int32_t* out_token, float* out_conf, float* out_lse,
+                   void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+    if (!hidden_bf16 || !w_lm_bf16 || !out_token || !out_conf || !workspace) return PSD_ERR_NULL;
+    if (row_ids) return PSD_ERR_UNSUPPORTED;
+    if (!conf_shape_ok(n_rows, H, V)) return PSD_ERR_SHAPE;
+    if (!aligned(hidden_bf16, 16) || !aligned(w_lm_bf16, 16) || !aligned(workspace, 256) ||
+        !aligned(out_token, 4) || !aligned(out_conf, 4) || !aligned(out_lse, 4) || !aligned(status_dev, 4))
+        return PSD_ERR_ALIGN;
+    if (workspace_bytes < psd_workspace_bytes(n_rows, H, V)) return PSD_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    Partials part = carve_partials(workspace, n_rows, V);
+    int n_split = g_conf_impl.load() == 1
+                      ? launch_confidence_simt(hidden_bf16, w_lm_bf16, n_rows, H, V, part, st)
+                      : launch_confidence_tc(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st);
+    if (n_split < 0) return n_split;
+    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st);
+}
+
+int psd_select_unmask(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
+                      int32_t* tokens, int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
+                      int32_t* sel, int32_t* n_sel, int32_t* sel_pos, void* cuda_stream) {
+    if (!conf || !tok || !tokens || !mask || !sel || !n_sel || !sel_pos) return PSD_ERR_NULL;
+    if (check_block_shape(B, M) || n_nodes < 1 || n_nodes > PSD_MAX_DEPTH) return PSD_ERR_SHAPE;
+    if (int e = check_policy(p)) return e;
+    return launch_select(conf, tok, node, n_nodes, tokens, mask, B, M, p, sel, n_sel, sel_pos,
+                         reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int psd_build_drafts(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
+                     const int32_t* tokens, const int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
+                     int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens, int32_t* draft_mask,
+                     void* cuda_stream) {
+    if (!conf || !tok || !tokens || !mask || !sigma || !n_fill || !draft_tokens || !draft_mask) return PSD_ERR_NULL;
+    if (check_block_shape(B, M) || n_nodes < 1 || n_nodes > PSD_MAX_DEPTH) return PSD_ERR_SHAPE;
+    if (int e = check_policy(p)) return e;
+    return launch_build(conf, tok, node, n_nodes, tokens, mask, B, M, p, sigma, n_fill, draft_tokens, draft_mask,
+                        reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+int psd_verify_accept(const int32_t* tokV, const float* confV, const int32_t* sigma, const int32_t* n_fill,
+                      const int32_t* draft_tokens, const int32_t* draft_mask, int32_t B, int32_t M, psd_policy_t p,
+                      int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec_accepted,
+                      int32_t* n_committed, int32_t* accepted, void* cuda_stream) {
+    if (!tokV || !confV || !sigma || !n_fill || !draft_tokens || !draft_mask || !tokens || !mask || !k_star ||
+        !n_spec_accepted || !n_committed)
+        return PSD_ERR_NULL;
+    if (check_block_shape(B, M)) return PSD_ERR_SHAPE;
+    if (int e = check_policy(p)) return e;
+    return launch_accept(tokV, confV, sigma, n_fill, draft_tokens, draft_mask, B, M, p, tokens, mask, k_star,
+                         n_spec_accepted, n_committed, accepted, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+static int check_step_io(const psd_step_io_t* io) {
+    if (!io) return PSD_ERR_NULL;
+    if (!io->hidden_bf16 || !io->w_lm_bf16 || !io->sigma || !io->n_fill || !io->draft_tokens || !io->draft_mask ||
+        !io->tokV || !io->confV || !io->tokens || !io->mask || !io->k_star || !io->n_spec_accepted ||
+        !io->n_committed || !io->sel || !io->n_sel || !io->sel_pos)
+        return PSD_ERR_NULL;
+    return PSD_OK;
+}
+
+int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+             void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+    if (int e = check_step_io(io)) return e;
+    if (check_block_shape(B, M)) return PSD_ERR_SHAPE;
+    if (int e = check_policy(p)) return e;
+    const int D = p.depth;
+    if ((long long)B * D * M > 2147483647ll) return PSD_ERR_SHAPE;
+    const int n_rows = B * D * M;
+    int e = psd_confidence(io->hidden_bf16, io->w_lm_bf16, nullptr, n_rows, H, V, io->tokV, io->confV, nullptr,
+                           workspace, workspace_bytes, status_dev, cuda_stream);
+    if (e) return e;
+    e = psd_verify_accept(io->tokV, io->confV, io->sigma, io->n_fill, io->draft_tokens, io->draft_mask, B, M, p,
+                          io->tokens, io->mask, io->k_star, io->n_spec_accepted, io->n_committed, nullptr,
+                          cuda_stream);
+    if (e) return e;
+    e = psd_select_unmask(io->confV, io->tokV, io->k_star, D, io->tokens, io->mask, B, M, p, io->sel, io->n_sel,
+                          io->sel_pos, cuda_stream);
+    if (e) return e;
+    return psd_build_drafts(io->confV, io->tokV, io->k_star, D, io->tokens, io->mask, B, M, p, io->sigma,
+                            io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream);
+}
+
+// Device staging layout of psd_step_host, in order; every piece 256-byte aligned.
+namespace {
+struct Staging {
+    size_t hidden, sigma, n_fill, draft_tokens, draft_mask, tokV, confV, tokens, mask, k_star, n_spec, n_comm,
+        sel, n_sel, sel_pos, status, workspace, total;
+};
+Staging staging_layout(int B, int M, int H, int V, int D) {
+    Staging s;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o += round_up(bytes, 256); return at; };
+    const size_t R = (size_t)B * D * M, BM = (size_t)B * M;
+    s.hidden = take(R * H * 2);
+    s.sigma = take(BM * 4);
+    s.n_fill = take((size_t)B * D * 4);
+    s.draft_tokens = take(R * 4);
+    s.draft_mask = take(R * 4);
+    s.tokV = take(R * 4);
+    s.confV = take(R * 4);
+    s.tokens = take(BM * 4);
+    s.mask = take(BM * 4);
+    s.k_star = take((size_t)B * 4);
+    s.n_spec = take((size_t)B * 4);
+    s.n_comm = take((size_t)B * 4);
+    s.sel = take(BM * 4);
+    s.n_sel = take((size_t)B * 4);
+    s.sel_pos = take(BM * 4);
+    s.status = take(4);
+    s.workspace = take(psd_workspace_bytes((int)R, H, V));
+    s.total = o;
+    return s;
+}
+}  // namespace
+
+size_t psd_step_host_bytes(int32_t B, int32_t M, int32_t H, int32_t V, int32_t D) {
+    if (check_block_shape(B, M) || D < 1 || D > PSD_MAX_DEPTH || (long long)B * D * M > 2147483647ll) return 0;
+    if (!conf_shape_ok(B * D * M, H, V)) return 0;
+    return staging_layout(B, M, H, V, D).total;
+}
+
+int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+                  void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream) {
+    if (int e = check_step_io(io)) return e;
+    if (!staging) return PSD_ERR_NULL;
+    if (check_block_shape(B, M)) return PSD_ERR_SHAPE;
+    if (int e = check_policy(p)) return e;
+    const int D = p.depth;
+    const size_t need = psd_step_host_bytes(B, M, H, V, D);
+    if (need == 0) return PSD_ERR_SHAPE;
+    if (!aligned(staging, 256)) return PSD_ERR_ALIGN;
+    if (staging_bytes < need) return PSD_ERR_WORKSPACE;
+    const Staging s = staging_layout(B, M, H, V, D);
+    unsigned char* d = reinterpret_cast<unsigned char*>(staging);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const size_t R = (size_t)B * D * M, BM = (size_t)B * M;
+    bool ok = true;
+    auto h2d = [&](size_t off, const void* src, size_t bytes) {
+        ok = ok && cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    };
+    auto d2h = [&](void* dst, size_t off, size_t bytes) {
+        ok = ok && cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    h2d(s.hidden, io->hidden_bf16, R * H * 2);
+    h2d(s.sigma, io->sigma, BM * 4);
+    h2d(s.n_fill, io->n_fill, (size_t)B * D * 4);
+    h2d(s.draft_tokens, io->draft_tokens, R * 4);
+    h2d(s.draft_mask, io->draft_mask, R * 4);
+    ok = ok && cudaMemsetAsync(d + s.status, 0, 4, st) == cudaSuccess;
+    if (!ok) return PSD_ERR_CUDA;
+
+    psd_step_io_t dev;
+    dev.hidden_bf16 = d + s.hidden;
+    dev.w_lm_bf16 = io->w_lm_bf16;
+    dev.sigma = reinterpret_cast<int32_t*>(d + s.sigma);
+    dev.n_fill = reinterpret_cast<int32_t*>(d + s.n_fill);
+    dev.draft_tokens = reinterpret_cast<int32_t*>(d + s.draft_tokens);
+    dev.draft_mask = reinterpret_cast<int32_t*>(d + s.draft_mask);
+    dev.tokV = reinterpret_cast<int32_t*>(d + s.tokV);
+    dev.confV = reinterpret_cast<float*>(d + s.confV);
+    dev.tokens = reinterpret_cast<int32_t*>(d + s.tokens);
+    dev.mask = reinterpret_cast<int32_t*>(d + s.mask);
+    dev.k_star = reinterpret_cast<int32_t*>(d + s.k_star);
+    dev.n_spec_accepted = reinterpret_cast<int32_t*>(d + s.n_spec);
+    dev.n_committed = reinterpret_cast<int32_t*>(d + s.n_comm);
+    dev.sel = reinterpret_cast<int32_t*>(d + s.sel);
+    dev.n_sel = reinterpret_cast<int32_t*>(d + s.n_sel);
+    dev.sel_pos = reinterpret_cast<int32_t*>(d + s.sel_pos);
+    int e = psd_step(&dev, B, M, H, V, p, d + s.workspace, need - s.workspace,
+                     reinterpret_cast<int32_t*>(d + s.status), cuda_stream);
+    if (e) return e;
+
+    d2h(io->sigma, s.sigma, BM * 4);
+    d2h(io->n_fill, s.n_fill, (size_t)B * D * 4);
+    d2h(io->draft_tokens, s.draft_tokens, R * 4);
+    d2h(io->draft_mask, s.draft_mask, R * 4);
+    d2h(io->tokV, s.tokV, R * 4);
+    d2h(io->confV, s.confV, R * 4);
+    d2h(io->tokens, s.tokens, BM * 4);
+    d2h(io->mask, s.mask, BM * 4);
+    d2h(io->k_star, s.k_star, (size_t)B * 4);
+    d2h(io->n_spec_accepted, s.n_spec, (size_t)B * 4);
+    d2h(io->n_committed, s.n_comm, (size_t)B * 4);
+    d2h(io->sel, s.sel, BM * 4);
+    d2h(io->n_sel, s.n_sel, (size_t)B * 4);
+    d2h(io->sel_pos, s.sel_pos, BM * 4);
+    int32_t status = 0;
+    ok = ok && cudaMemcpyAsync(&status, d + s.status, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) return PSD_ERR_CUDA;
+    if (status_host) *status_host = status;
+    return PSD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,59 @@
+// Internal declarations shared by the translation units of libpsd_b200 (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "psd.h"
+
+namespace psd {
+
+// Width (vocabulary entries) of one split of the vocabulary in the tensor-core kernel; the
+// workspace is sized for one partial triple per (row, split) at this granularity or coarser.
+constexpr int kMinSplitWidth = 128;
+
+// Workspace layout: three arrays [n_split][n_rows] (max, sum-exp, argmax), n_split <= max_splits(V).
+inline int max_splits(int V) { return (V + kMinSplitWidth - 1) / kMinSplitWidth; }
+
+struct Partials {
+    float* m;      // [n_split][n_rows] running max of the split's logits
+    float* s;      // [n_split][n_rows] sum of exp(l - m) over the split
+    int32_t* a;    // [n_split][n_rows] lowest vocabulary index attaining m
+};
+
+inline Partials carve_partials(void* workspace, int n_rows, int V) {
+    size_t n = (size_t)max_splits(V) * (size_t)n_rows;
+    Partials p;
+    p.m = reinterpret_cast<float*>(workspace);
+    p.s = p.m + n;
+    p.a = reinterpret_cast<int32_t*>(p.s + n);
+    return p;
+}
+
+void count_launch(int n = 1);
+
+// confidence_simt.cu: plain CUDA-core kernel. Returns the number of splits written, or < 0.
+int launch_confidence_simt(const void* hidden, const void* w, int n_rows, int H, int V,
+                           Partials part, cudaStream_t st);
+
+// confidence_tc.cu: tcgen05 + TMA kernel. Returns the number of splits written, or < 0 (psd_status).
+int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V,
+                         Partials part, int32_t* status_dev, cudaStream_t st);
+
+// combine.cu: merge n_split partial triples per row.
+int launch_combine(Partials part, int n_split, int n_rows,
+                   int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st);
+
+// policy.cu
+int launch_select(const float* conf, const int32_t* tok, const int32_t* node, int n_nodes,
+                  int32_t* tokens, int32_t* mask, int B, int M, psd_policy_t p,
+                  int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st);
+int launch_build(const float* conf, const int32_t* tok, const int32_t* node, int n_nodes,
+                 const int32_t* tokens, const int32_t* mask, int B, int M, psd_policy_t p,
+                 int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens, int32_t* draft_mask,
+                 cudaStream_t st);
+int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma, const int32_t* n_fill,
+                  const int32_t* draft_tokens, const int32_t* draft_mask, int B, int M, psd_policy_t p,
+                  int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec, int32_t* n_comm,
+                  int32_t* accepted, cudaStream_t st);
+
+}  // namespace psd

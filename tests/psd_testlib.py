@@ -1,0 +1,182 @@
+"""Shared helpers of the GPU parity tests: upload seeded inputs, call the C-ABI through the binding,
+and compare with the CPU oracle under the stated tolerances."""
+from __future__ import annotations
+
+import functools
+
+import numpy as np
+import torch
+
+import oracle
+import paper_2605_15609_b200 as psd
+import psd_inputs as gen
+
+CONF_ATOL = 2e-3   # absolute tolerance on confidences
+GAP_MIN = 1e-2     # rows whose top-1/top-2 logit gap is below this are set aside for the token check
+TAU_MARGIN = 1e-3  # free-running chains: a confidence this close to tau makes its block a near-tie
+RANK_MARGIN = 5e-5 # ... and so do two confidences of one node within this relative distance
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def bf16_dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+@functools.lru_cache(maxsize=2)
+def weights_cached(name):
+    cfg = gen.CONFIGS[name]
+    W = gen.weights(cfg)
+    return W, bf16_dev(W)
+
+
+def f32(x) -> float:
+    return float(np.float32(x))
+
+
+def policies(cfg: gen.Config, D=None, accept_mode=0):
+    """The same policy for the oracle and for the library; tau is the fp32 value on both sides."""
+    D = cfg.D if D is None else D
+    tau = f32(cfg.tau)
+    po = oracle.Policy(tau=tau, k_min=cfg.k_min, k_max=cfg.k_max, depth=D, stride=cfg.stride,
+                       accept_mode=accept_mode, mask_id=cfg.mask_id)
+    pg = psd.policy(tau=tau, k_min=cfg.k_min, k_max=cfg.k_max, depth=D, stride=cfg.stride,
+                    accept_mode=accept_mode, mask_id=cfg.mask_id)
+    return po, pg
+
+
+def gpu_confidence(hidden_dev, w_dev, want_lse=True, impl=0):
+    n, H = hidden_dev.shape
+    V = w_dev.shape[0]
+    tok = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+    conf = torch.full((n,), -7.0, dtype=torch.float32, device="cuda")
+    lse = torch.full((n,), -7.0, dtype=torch.float32, device="cuda") if want_lse else None
+    ws = torch.empty(psd.psd_workspace_bytes(n, H, V), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    prev = psd.psd_set_confidence_impl(impl)
+    try:
+        psd.psd_confidence(hidden_dev, w_dev, tok, conf, lse, ws, status)
+        torch.cuda.synchronize()
+    finally:
+        psd.psd_set_confidence_impl(prev)
+    assert int(status.item()) == 0, psd.status_string(int(status.item()))
+    return tok.cpu().numpy(), conf.cpu().numpy(), (lse.cpu().numpy() if want_lse else None)
+
+
+def check_confidence(tok_g, conf_g, lse_g, tok_o, conf_o, lse_o, gap_o):
+    """Token ids bit-exact on rows with a clear winner; confidences within CONF_ATOL on every row.
+    Returns the number of rows set aside for the token check."""
+    assert np.isfinite(conf_g).all()
+    err = np.abs(conf_g.astype(np.float64) - conf_o)
+    assert err.max() <= CONF_ATOL, f"max |conf - oracle| = {err.max():.3e}"
+    clear = gap_o >= GAP_MIN
+    bad = np.nonzero(clear & (tok_g != tok_o))[0]
+    assert bad.size == 0, f"token mismatch on rows {bad[:8]} (gaps {gap_o[bad[:8]]})"
+    if lse_g is not None:
+        assert np.abs(lse_g.astype(np.float64) - lse_o).max() <= 2e-3
+    return int((~clear).sum())
+
+
+class GpuChain:
+    """Device buffers for the three integer stages of B blocks."""
+
+    def __init__(self, B, M, D):
+        i32 = lambda *s: torch.full(s, -9, dtype=torch.int32, device="cuda")
+        self.B, self.M, self.D = B, M, D
+        self.sel, self.n_sel, self.sel_pos = i32(B, M), i32(B), i32(B, M)
+        self.sigma, self.n_fill = i32(B, M), i32(B, D)
+        self.draft_tokens, self.draft_mask = i32(B, D, M), i32(B, D, M)
+        self.k_star, self.n_spec, self.n_comm, self.accepted = i32(B), i32(B), i32(B), i32(B, D)
+        self.tokens_out, self.mask_out = i32(B, M), i32(B, M)
+
+
+def np_(t):
+    return t.cpu().numpy()
+
+
+# ----------------------------------------------------------------------------------------------
+# Whole-step chains: prologue (stage-1 pass -> policy -> drafts) and the step itself
+# (verification pass -> acceptance -> policy on node k* -> drafts for the next step).
+# ----------------------------------------------------------------------------------------------
+
+def gpu_prologue(cfg, h1_dev, w_dev, pg):
+    """psd_confidence on the stage-1 rows, then psd_select_unmask and psd_build_drafts from a fully
+    masked block.  Returns a dict of numpy outputs and the device StepBuffers ready for psd_step."""
+    B, M, D = cfg.B, cfg.M, cfg.D
+    tok1, conf1, _ = gpu_confidence(h1_dev, w_dev, want_lse=False)
+    g = GpuChain(B, M, D)
+    tokens = torch.full((B, M), cfg.mask_id, dtype=torch.int32, device="cuda")
+    mask = torch.ones((B, M), dtype=torch.int32, device="cuda")
+    c1, t1 = dev(conf1.reshape(B, 1, M)), dev(tok1.reshape(B, 1, M))
+    psd.psd_select_unmask(c1, t1, tokens, mask, pg, g.sel, g.n_sel, g.sel_pos)
+    psd.psd_build_drafts(c1, t1, tokens, mask, pg, g.sigma, g.n_fill, g.draft_tokens, g.draft_mask)
+    torch.cuda.synchronize()
+    out = dict(tok1=tok1.reshape(B, M), conf1=conf1.reshape(B, M), tokens=np_(tokens), mask=np_(mask),
+               sel=np_(g.sel), n_sel=np_(g.n_sel), sel_pos=np_(g.sel_pos), sigma=np_(g.sigma),
+               n_fill=np_(g.n_fill), draft_tokens=np_(g.draft_tokens), draft_mask=np_(g.draft_mask))
+    return out, g
+
+
+def oracle_prologue(cfg, tok1, conf1, po):
+    B, M = cfg.B, cfg.M
+    tokens = np.full((B, M), cfg.mask_id, dtype=np.int32)
+    mask = np.ones((B, M), dtype=np.int32)
+    tokens, mask, sel, n_sel, sel_pos = oracle.select_unmask(conf1, tok1, tokens, mask, po)
+    sigma, n_fill, dt, dm = oracle.build_drafts(conf1, tok1, tokens, mask, po)
+    return dict(tokens=tokens, mask=mask, sel=sel, n_sel=n_sel, sel_pos=sel_pos, sigma=sigma, n_fill=n_fill,
+                draft_tokens=dt, draft_mask=dm)
+
+
+def oracle_step(cfg, tokV, confV, pro, po):
+    """The step on given verifier outputs [B, D, M]: accept -> policy on node k* -> next drafts."""
+    B = cfg.B
+    tokens, mask, k_star, n_spec, n_comm, acc = oracle.verify_accept(
+        tokV, confV, pro["sigma"], pro["n_fill"], pro["draft_tokens"], pro["draft_mask"], po)
+    rows = np.arange(B)
+    ck, tk = confV[rows, k_star], tokV[rows, k_star]
+    tokens2, mask2, sel, n_sel, sel_pos = oracle.select_unmask(ck, tk, tokens, mask, po)
+    sigma, n_fill, dt, dm = oracle.build_drafts(ck, tk, tokens2, mask2, po)
+    return dict(k_star=k_star, n_spec_accepted=n_spec, n_committed=n_comm, tokens=tokens2, mask=mask2, sel=sel,
+                n_sel=n_sel, sel_pos=sel_pos, sigma=sigma, n_fill=n_fill, draft_tokens=dt, draft_mask=dm)
+
+
+STEP_INT_OUTPUTS = ("k_star", "n_spec_accepted", "n_committed", "tokens", "mask", "sel", "n_sel", "sel_pos",
+                    "sigma", "n_fill", "draft_tokens", "draft_mask")
+
+
+def step_buffers_from(g: GpuChain, cfg, hidden_dev, w_dev):
+    B, M, D = cfg.B, cfg.M, cfg.D
+    buf = psd.StepBuffers.allocate(B, M, D, cfg.H, hidden_dev, w_dev, "cuda")
+    buf.sigma.copy_(g.sigma)
+    buf.n_fill.copy_(g.n_fill)
+    buf.draft_tokens.copy_(g.draft_tokens)
+    buf.draft_mask.copy_(g.draft_mask)
+    return buf
+
+
+def gpu_step(buf, cfg, pg):
+    ws = torch.empty(psd.psd_workspace_bytes(cfg.rows, cfg.H, cfg.V), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    psd.psd_step(buf, pg, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    out = {k: np_(getattr(buf, k)) for k in STEP_INT_OUTPUTS}
+    out["tokV"], out["confV"] = np_(buf.tokV), np_(buf.confV)
+    return out
+
+
+def threshold_margin_ok(conf_rows, tau):
+    """No confidence of the group is within TAU_MARGIN of tau."""
+    return bool(np.abs(np.asarray(conf_rows, dtype=np.float64) - tau).min() >= TAU_MARGIN)
+
+
+def ranking_margin_ok(conf_rows):
+    """No two confidences of the group are within a relative RANK_MARGIN (the fp32 path's relative
+    error on a confidence is about 3e-5: fp32 accumulation over H plus the exponential)."""
+    c = np.sort(np.asarray(conf_rows, dtype=np.float64))
+    return bool((np.diff(c) > RANK_MARGIN * c[1:]).all())
