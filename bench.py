@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the PSD per-step hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+A step is one pass of the whole path over one batch of synthetic input: psd_confidence on all
+B*D*M rows of the verification batch, then psd_verify_accept, psd_select_unmask and
+psd_build_drafts (psd_step), on one stream.  The metric is masked positions scored and accepted
+per second = B*D*M / t_step.  Rank 0 prints ONE JSON line.
+
+For N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
+replica on its own batch: no data-path collective, weak scaling.
+
+--impl reference times the CPU oracle (the only "reference implementation" of this path) on the
+host cores, on bounded samples of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "masked positions scored+accepted/sec per step"
+UNIT = "positions/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel, from the ncu captures
+# summarised under profiles/ (None where no capture of that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._period = period_s
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def sample(self):
+        if self._nv is None:
+            return
+        try:
+            mhz = int(self._nv.nvmlDeviceGetClockInfo(self._h, self._nv.NVML_CLOCK_SM))
+            bits = int(self._nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+        except Exception:
+            return
+        self.samples.append(mhz)
+        for bit, name in self.REASONS.items():
+            if bits & bit:
+                self.reasons.add(name)
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample()
+            self._stop.wait(self._period)
+
+    def start(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def algorithmic_bytes(cfg) -> float:
+    """Bytes the method has to move per launch of the fused kernel: W once, the hidden rows once,
+    and 12 bytes of result per row.  Logits are not counted: the method never materialises them."""
+    R = cfg.rows
+    return float(cfg.V) * cfg.H * 2 + float(R) * cfg.H * 2 + 12.0 * R
+
+
+def algorithmic_flops(cfg) -> float:
+    return 2.0 * cfg.rows * cfg.V * cfg.H
+
+
+def ridge_rows(peaks) -> float:
+    return peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+
+
+# ------------------------------------------------------------------------------------ reference arm
+
+def oracle_sample_rate(cfg, wl, n_rows):
+    """Times the oracle on the first n_rows rows of the verification batch; returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    oracle.confidence(wl.hidden_verify[:n_rows], wl.W)
+    return time.perf_counter() - t0
+
+
+def oracle_full_step(cfg, wl, n_blocks, po):
+    """The oracle's whole step on the first n_blocks blocks: stage-1 pass, policy, drafts,
+    verification pass, acceptance, policy on node k*, next drafts.  Returns (seconds of the step
+    proper, rows scored by the step)."""
+    import oracle
+    B, M, D = n_blocks, cfg.M, cfg.D
+    tok1, conf1, _, _ = oracle.confidence(wl.hidden_stage1[:B * M], wl.W)
+    tokens = np.full((B, M), cfg.mask_id, dtype=np.int32)
+    mask = np.ones((B, M), dtype=np.int32)
+    tokens, mask, *_ = oracle.select_unmask(conf1.reshape(B, M), tok1.reshape(B, M), tokens, mask, po)
+    sigma, n_fill, dt, dm = oracle.build_drafts(conf1.reshape(B, M), tok1.reshape(B, M), tokens, mask, po)
+    t0 = time.perf_counter()
+    tokV, confV, _, _ = oracle.confidence(wl.hidden_verify[:B * D * M], wl.W)
+    tokV, confV = tokV.reshape(B, D, M), confV.reshape(B, D, M)
+    tokens, mask, ks, _, _, _ = oracle.verify_accept(tokV, confV, sigma, n_fill, dt, dm, po)
+    rows = np.arange(B)
+    tokens, mask, *_ = oracle.select_unmask(confV[rows, ks], tokV[rows, ks], tokens, mask, po)
+    oracle.build_drafts(confV[rows, ks], tokV[rows, ks], tokens, mask, po)
+    return time.perf_counter() - t0, B * D * M
+
+
+def oracle_policy(cfg):
+    import oracle
+    return oracle.Policy(tau=float(np.float32(cfg.tau)), k_min=cfg.k_min, k_max=cfg.k_max, depth=cfg.D,
+                         stride=cfg.stride, mask_id=cfg.mask_id)
+
+
+def cpu_baseline(cfg, wl, budget_s=15.0):
+    """The oracle as it stands, on the host cores, on a bounded sample of the workload."""
+    import oracle
+    probe_rows = min(4, cfg.rows)
+    t_probe = oracle_sample_rate(cfg, wl, probe_rows)
+    per_row = t_probe / probe_rows
+    rows_per_block = cfg.D * cfg.M
+    n_blocks = int(max(1, min(cfg.B, budget_s / max(per_row * rows_per_block, 1e-9))))
+    secs, rows = oracle_full_step(cfg, wl, n_blocks, oracle_policy(cfg))
+    return {"value": rows / secs, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"whole step on the first {n_blocks} of {cfg.B} blocks ({rows} of {cfg.rows} rows, "
+                      f"all {cfg.V} vocabulary entries), {secs:.2f} s"}
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle, K timed steps, each a bounded sample of the workload."""
+    import oracle
+    import psd_inputs as gen
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    wl = gen.make(cfg)
+    t_probe = oracle_sample_rate(cfg, wl, 1)
+    total_budget = 150.0
+    rows_per_step = int(max(1, min(cfg.rows, total_budget / max(t_probe, 1e-9) / (args.steps + args.warmup))))
+    rows_per_block = cfg.D * cfg.M
+    po = oracle_policy(cfg)
+    whole_blocks = rows_per_step >= rows_per_block
+    n_blocks = min(cfg.B, rows_per_step // rows_per_block) if whole_blocks else 0
+
+    def one_step():
+        if whole_blocks:
+            return oracle_full_step(cfg, wl, n_blocks, po)
+        t0 = time.perf_counter()
+        oracle.confidence(wl.hidden_verify[:rows_per_step], wl.W)
+        return time.perf_counter() - t0, rows_per_step
+
+    for _ in range(args.warmup):
+        one_step()
+    secs = rows = 0.0
+    for _ in range(args.steps):
+        s, r = one_step()
+        secs += s
+        rows += r
+    value = rows / secs
+    sample = (f"each step = the whole oracle step on {n_blocks} block(s)" if whole_blocks else
+              f"each step = the oracle's confidence computation on {rows_per_step} row(s) "
+              f"(fewer than one block of {rows_per_block}; the integer stages need whole blocks)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "D": cfg.D, "M": cfg.M, "H": cfg.H, "V": cfg.V,
+                       "rows_per_step": int(rows / args.steps)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------ our arm
+
+def run_ours(args, cfg):
+    import torch
+
+    import paper_2605_15609_b200 as psd
+    import psd_inputs as gen
+    from paper_2605_15609_b200 import replicas
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    info = replicas.rank_info_from_env()
+    torch.cuda.set_device(info.local_rank)
+    device = torch.device("cuda", info.local_rank)
+    replicas.init_process_group(info)
+    peaks, peaks_kind = load_peaks()
+
+    # Every replica holds the same W; each rank has its own batch of blocks.
+    W = gen.weights(cfg)
+    wl = gen.make(replace(cfg, seed=replicas.replica_seed(cfg.seed, info.rank)), W)
+    B, M, D, H, V, R = cfg.B, cfg.M, cfg.D, cfg.H, cfg.V, cfg.rows
+    pg = psd.policy(tau=float(np.float32(cfg.tau)), k_min=cfg.k_min, k_max=cfg.k_max, depth=D, stride=cfg.stride,
+                    mask_id=cfg.mask_id)
+
+    def bf16(bits, pin=False):
+        t = torch.from_numpy(bits.view(np.int16))
+        if pin:
+            return t.pin_memory().view(torch.bfloat16)
+        return t.to(device).view(torch.bfloat16)
+
+    w_dev, h1_dev, hv_dev = bf16(wl.W), bf16(wl.hidden_stage1), bf16(wl.hidden_verify)
+    ws = torch.empty(psd.psd_workspace_bytes(R, H, V), dtype=torch.uint8, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    stream = torch.cuda.current_stream()
+
+    # Untimed prologue: stage-1 pass -> policy -> first drafts.
+    buf = psd.StepBuffers.allocate(B, M, D, H, hv_dev, w_dev, device)
+    tok1 = torch.zeros(B * M, dtype=torch.int32, device=device)
+    conf1 = torch.zeros(B * M, dtype=torch.float32, device=device)
+    psd.psd_confidence(h1_dev, w_dev, tok1, conf1, None, ws, status)
+    buf.tokens.fill_(cfg.mask_id)
+    buf.mask.fill_(1)
+    c1, t1 = conf1.view(B, 1, M), tok1.view(B, 1, M)
+    psd.psd_select_unmask(c1, t1, buf.tokens, buf.mask, pg, buf.sel, buf.n_sel, buf.sel_pos)
+    psd.psd_build_drafts(c1, t1, buf.tokens, buf.mask, pg, buf.sigma, buf.n_fill, buf.draft_tokens, buf.draft_mask)
+    torch.cuda.synchronize()
+    first = {k: getattr(buf, k).clone() for k in ("sigma", "n_fill", "draft_tokens", "draft_mask")}
+
+    def timed_region(step_fn, n):
+        replicas.barrier(info, device)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(n):
+            step_fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        replicas.barrier(info, device)
+        return e0.elapsed_time(e1) * 1e-3
+
+    # ---- device-resident steps: the headline value
+    for _ in range(args.warmup):
+        psd.psd_step(buf, pg, ws, status, stream)
+    sampler = ClockSampler(physical_gpu_index(info.local_rank))
+    launches0 = psd.psd_launch_count()
+    sampler.start()
+    secs = timed_region(lambda i: psd.psd_step(buf, pg, ws, status, stream), args.steps)
+    sampler.sample()
+    sampler.stop()
+    launches = psd.psd_launch_count() - launches0
+    if int(status.item()) != 0:
+        raise RuntimeError("device status: " + psd.status_string(int(status.item())))
+    value, secs_max = replicas.aggregate_throughput(float(R) * args.steps, secs, info, device)
+
+    if args.profile_only:
+        if info.is_main:
+            print(json.dumps({"profile_only": True, "workload": cfg.name, "ms_per_step": 1e3 * secs_max / args.steps,
+                              "gpu_launches": launches}), flush=True)
+        return 0
+
+    # ---- the same region again with an event pair around the fused kernel of every step
+    n_k = min(args.steps, 512)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
+    for a, b in evs:          # torch creates the CUDA event on first record; the library re-records it later
+        a.record(stream)
+        b.record(stream)
+
+    def instrumented(i):
+        psd.psd_set_kernel_events(*evs[i])
+        psd.psd_step(buf, pg, ws, status, stream)
+
+    secs_instr = timed_region(instrumented, n_k)
+    kernel_ms = [a.elapsed_time(b) for a, b in evs]
+    kernel_s = statistics.fmean(kernel_ms) * 1e-3
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
+    hv_host = bf16(wl.hidden_verify, pin=True)
+    hb = psd.StepBuffers.allocate(B, M, D, H, hv_host, w_dev, "cpu", pin=True)
+    for k, v in first.items():
+        getattr(hb, k).copy_(v)
+    staging = torch.empty(psd.psd_step_host_bytes(B, M, H, V, D), dtype=torch.uint8, device=device)
+    n_e2e = max(3, min(args.steps, 200))
+    for _ in range(3):
+        psd.psd_step_host(hb, pg, staging, stream)
+    secs_e2e = timed_region(lambda i: psd.psd_step_host(hb, pg, staging, stream), n_e2e)
+    e2e_value, _ = replicas.aggregate_throughput(float(R) * n_e2e, secs_e2e, info, device)
+    h2d = R * H * 2 + 4 * (B * M + B * D + 2 * R)
+    d2h = 4 * (B * M + B * D + 2 * R) + 4 * (2 * R) + 4 * (2 * B * M) + 4 * (3 * B) + 4 * (2 * B * M + B) + 4
+
+    if not info.is_main:
+        return 0
+
+    tensor_bound = R > ridge_rows(peaks)
+    if tensor_bound:
+        peak = peaks["bf16_tflops_sustained"] if secs_max > 1.0 else peaks["bf16_tflops"]
+        achieved = algorithmic_flops(cfg) / kernel_s / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_kind": f"{'sustained' if secs_max > 1.0 else 'burst'} bf16, of {peaks_kind}",
+                "frac_of_burst": achieved / peaks["bf16_tflops"]}
+    else:
+        peak = peaks["hbm_gbs"]
+        achieved = algorithmic_bytes(cfg) / kernel_s / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"copy bandwidth, of {peaks_kind}"}
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(cfg.name)
+    roof["kernel"] = "confidence_tc_kernel"
+    roof["kernel_ms"] = kernel_s * 1e3
+    roof["kernel_launches_timed"] = n_k
+    roof["step_ms_while_instrumented"] = 1e3 * secs_instr / n_k
+    roof["algorithmic_bytes"] = algorithmic_bytes(cfg)
+    roof["algorithmic_flops"] = algorithmic_flops(cfg)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": info.world_size, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * secs_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": B, "D": D, "M": M, "H": H, "V": V, "rows": R,
+                       "policy": {"tau": cfg.tau, "k_min": cfg.k_min, "k_max": cfg.k_max, "stride": cfg.stride},
+                       "parallelism": f"replicas x{info.world_size}",
+                       "l2": f"inputs larger than L2: W is {V * H * 2 / 1e6:.0f} MB and is re-read every step"},
+            "clocks": sampler.summary(),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": 1e3 * secs_e2e / n_e2e, "steps": n_e2e},
+            "gpu_launches": launches,
+            "roofline": roof,
+            "cpu_baseline": cpu_baseline(cfg, wl)}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", default="single_request",
+                    help="workload: tiny, single_request, class_7b, batched_serving, deep_sweep[_D1|_D2|_D4]")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile-only", action="store_true",
+                    help="for runs under a profiler: device-resident steps only (no instrumented pass, no "
+                         "end-to-end pass, no CPU baseline); the printed line is not a benchmark result")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    import psd_inputs as gen
+    name = args.config
+    if name.startswith("deep_sweep_D"):
+        cfg = gen.with_depth(gen.CONFIGS["deep_sweep"], int(name.rsplit("D", 1)[1]))
+    else:
+        cfg = gen.CONFIGS[name]
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+    return run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

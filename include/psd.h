@@ -234,6 +234,15 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
  */
 int psd_set_confidence_impl(int impl);
 
+/*
+ * Profiling aid.  When both events (cudaEvent_t passed as void*) are non-NULL, the next
+ * psd_confidence call made by this host thread (directly or through psd_step / psd_step_host)
+ * records `start_event` immediately before and `stop_event` immediately after its main kernel
+ * (the fused LM-head + confidence kernel, not the combine pass) on the call's stream; the hook then
+ * clears itself.  Passing NULLs clears it.  Always returns PSD_OK.
+ */
+int psd_set_kernel_events(void* start_event, void* stop_event);
+
 /* Number of kernel launches the library has issued in this process (all entry points). */
 int64_t psd_launch_count(void);
 

@@ -70,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.psd_step_host.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
     lib.psd_set_confidence_impl.restype = ctypes.c_int
     lib.psd_set_confidence_impl.argtypes = [ctypes.c_int]
+    lib.psd_set_kernel_events.restype = ctypes.c_int
+    lib.psd_set_kernel_events.argtypes = [_vp, _vp]
     lib.psd_launch_count.restype = _i64
     lib.psd_launch_count.argtypes = []
     return lib
@@ -113,6 +115,15 @@ def psd_workspace_bytes(n_rows: int, H: int, V: int) -> int:
 
 def psd_set_confidence_impl(impl: int) -> int:
     return int(LIB.psd_set_confidence_impl(int(impl)))
+
+
+def psd_set_kernel_events(start_event, stop_event) -> int:
+    """torch.cuda.Event objects (already recorded once or created with enable_timing=True), or None."""
+    def h(e):
+        if e is None:
+            return None
+        return e.cuda_event if hasattr(e, "cuda_event") else int(e)
+    return int(LIB.psd_set_kernel_events(h(start_event), h(stop_event)))
 
 
 def psd_launch_count() -> int:

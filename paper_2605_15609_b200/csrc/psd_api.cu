@@ -8,6 +8,7 @@ namespace psd {
 namespace {
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_conf_impl{0};
+thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -58,6 +59,12 @@ int psd_set_confidence_impl(int impl) {
     return g_conf_impl.exchange(impl);
 }
 
+int psd_set_kernel_events(void* start_event, void* stop_event) {
+    t_ev_start = reinterpret_cast<cudaEvent_t>(start_event);
+    t_ev_stop = reinterpret_cast<cudaEvent_t>(stop_event);
+    return PSD_OK;
+}
+
 int64_t psd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_ids,
@@ -73,9 +80,16 @@ int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t
     if (workspace_bytes < psd_workspace_bytes(n_rows, H, V)) return PSD_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     Partials part = carve_partials(workspace, n_rows, V);
+    const bool timed = t_ev_start && t_ev_stop;
+    if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
     int n_split = g_conf_impl.load() == 1
                       ? launch_confidence_simt(hidden_bf16, w_lm_bf16, n_rows, H, V, part, st)
                       : launch_confidence_tc(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st);
+    if (timed) {
+        cudaError_t e = cudaEventRecord(t_ev_stop, st);
+        t_ev_start = t_ev_stop = nullptr;
+        if (e != cudaSuccess) return PSD_ERR_CUDA;
+    }
     if (n_split < 0) return n_split;
     return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st);
 }
