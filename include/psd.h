@@ -177,6 +177,35 @@ int psd_verify_accept(const int32_t* tokV, const float* confV,
                       int32_t* accepted, void* cuda_stream);
 
 /*
+ * psd_confidence_static — psd_confidence without a workspace argument and without any allocation.
+ * (The paper has no counterpart: this entry point exists for deployment, not for the method.)
+ *
+ * For callers that cannot allocate device memory at the point of the call — a server whose own
+ * pool already owns all free HBM, a plug-in invoked from another runtime's callback where
+ * cudaMalloc and its implicit synchronisation are not allowed.  The scratch that psd_confidence
+ * takes from its caller lives here in a fixed array inside the library image, of
+ * PSD_STATIC_SCRATCH_BYTES; every GPU that loads the library holds that much until the process exits.
+ *
+ * Same arguments, outputs and numerics as psd_confidence (always the tcgen05 kernel), except:
+ *   - no workspace; sizes with psd_workspace_bytes(n_rows, H, V) > PSD_STATIC_SCRATCH_BYTES are
+ *     rejected with PSD_ERR_WORKSPACE (e.g. 128 rows x V = 126464 needs 1.5 MB and fits;
+ *     8192 rows do not);
+ *   - the first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current); make that first call outside of any
+ *     stream capture;
+ *   - it calls no cudaMalloc, cudaFree or other allocating routine;
+ *   - all calls on a device share the one array, which keeps the previous call's contents.
+ *     Nothing in it needs clearing (every entry read is written first by the same call), but two
+ *     calls that overlap on the GPU (different streams, or different host threads) race on it:
+ *     serialise them.
+ */
+#define PSD_STATIC_SCRATCH_BYTES (4u << 20)
+int psd_confidence_static(const void* hidden_bf16, const void* w_lm_bf16,
+                          int32_t n_rows, int32_t H, int32_t V,
+                          int32_t* out_token, float* out_conf, float* out_lse,
+                          int32_t* status_dev, void* cuda_stream);
+
+/*
  * All pointers of one decoding step over a batch of B blocks.  Device pointers for psd_step,
  * HOST pointers (pinned memory recommended) for psd_step_host, except w_lm_bf16 which is a
  * device pointer in both.

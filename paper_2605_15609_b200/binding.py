@@ -55,6 +55,8 @@ def _load() -> ctypes.CDLL:
     lib.psd_workspace_bytes.argtypes = [_i32, _i32, _i32]
     lib.psd_confidence.restype = ctypes.c_int
     lib.psd_confidence.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    lib.psd_confidence_static.restype = ctypes.c_int
+    lib.psd_confidence_static.argtypes = [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
     lib.psd_select_unmask.restype = ctypes.c_int
     lib.psd_select_unmask.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, pol, _vp, _vp, _vp, _vp]
     lib.psd_build_drafts.restype = ctypes.c_int
@@ -139,6 +141,19 @@ def psd_confidence(hidden, w_lm, out_token, out_conf, out_lse=None, workspace=No
     _check(LIB.psd_confidence(_ptr(hidden), _ptr(w_lm), _ptr(row_ids), n_rows, H, V, _ptr(out_token),
                               _ptr(out_conf), _ptr(out_lse), _ptr(workspace), ws_bytes, _ptr(status),
                               _stream(stream)), "psd_confidence")
+
+
+PSD_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def psd_confidence_static(hidden, w_lm, out_token, out_conf, out_lse=None, status=None, stream=None):
+    """psd_confidence for callers that cannot allocate: the scratch is a fixed array inside the
+    library (PSD_STATIC_SCRATCH_BYTES); larger problems raise PSD_ERR_WORKSPACE.  Calls on one device
+    must not overlap."""
+    n_rows, H = hidden.shape
+    _check(LIB.psd_confidence_static(_ptr(hidden), _ptr(w_lm), n_rows, H, w_lm.shape[0], _ptr(out_token),
+                                     _ptr(out_conf), _ptr(out_lse), _ptr(status), _stream(stream)),
+           "psd_confidence_static")
 
 
 def psd_select_unmask(conf, tok, tokens, mask, p: PsdPolicy, sel, n_sel, sel_pos, node=None, n_nodes=1,
