@@ -264,6 +264,15 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
 int psd_set_confidence_impl(int impl);
 
 /*
+ * Performance knobs (process-wide; results never depend on them).  Returns PSD_OK,
+ * PSD_ERR_UNSUPPORTED for an unknown knob or PSD_ERR_SHAPE for a bad value.
+ *   PSD_TUNE_BAND_BYTES  bytes of W that one band of the fused kernel's tile order may hold in L2
+ *                        (default 16 MiB); 0 means one vocabulary tile per band
+ */
+#define PSD_TUNE_BAND_BYTES 1
+int psd_set_tuning(int knob, int value);
+
+/*
  * Profiling aid.  When both events (cudaEvent_t passed as void*) are non-NULL, the next
  * psd_confidence call made by this host thread (directly or through psd_step / psd_step_host)
  * records `start_event` immediately before and `stop_event` immediately after its main kernel

@@ -72,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.psd_step_host.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
     lib.psd_set_confidence_impl.restype = ctypes.c_int
     lib.psd_set_confidence_impl.argtypes = [ctypes.c_int]
+    lib.psd_set_tuning.restype = ctypes.c_int
+    lib.psd_set_tuning.argtypes = [ctypes.c_int, ctypes.c_int]
     lib.psd_set_kernel_events.restype = ctypes.c_int
     lib.psd_set_kernel_events.argtypes = [_vp, _vp]
     lib.psd_launch_count.restype = _i64
@@ -117,6 +119,13 @@ def psd_workspace_bytes(n_rows: int, H: int, V: int) -> int:
 
 def psd_set_confidence_impl(impl: int) -> int:
     return int(LIB.psd_set_confidence_impl(int(impl)))
+
+
+PSD_TUNE_BAND_BYTES = 1
+
+
+def psd_set_tuning(knob: int, value: int) -> int:
+    return int(LIB.psd_set_tuning(int(knob), int(value)))
 
 
 def psd_set_kernel_events(start_event, stop_event) -> int:

@@ -1,0 +1,63 @@
+// Device-side merge of per-split (max, sum-exp, argmax) triples, shared by the stand-alone combine
+// kernel and by the fused step-tail kernel so that both produce bitwise identical results.
+#pragma once
+#include "psd_internal.cuh"
+
+namespace psd {
+
+struct Triple {
+    float m, s;
+    int32_t a;
+};
+
+__device__ __forceinline__ void merge_triple(Triple& x, float m, float s, int32_t a) {
+    if (m > x.m) {
+        x.s = x.s * expf(x.m - m) + s;
+        x.m = m;
+        x.a = a;
+    } else if (m == x.m) {
+        x.s += s;
+        x.a = min(x.a, a);
+    } else {
+        x.s += s * expf(m - x.m);   // also the NaN path: the sum becomes NaN and stays NaN
+    }
+}
+
+constexpr int kCombineRows = 32;   // rows handled by one group of threads
+constexpr int kCombineLanes = 8;   // threads per row
+constexpr int kCombineThreads = kCombineRows * kCombineLanes;
+
+// One group of 256 threads (g = 0..255 within the group) merges the splits of rows
+// row0 .. row0+31: thread (lane = g / 32, tx = g % 32) walks splits lane, lane+8, ... of row
+// row0 + tx (a warp reads 32 consecutive rows of one split: coalesced), then lane 0 merges the 8
+// partial results of its row in lane order.  `sh` is this group's scratch [8][32].
+// Every thread of the group must call this (it synchronises the whole block twice).
+__device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, const float* __restrict__ ps,
+                                               const int32_t* __restrict__ pa, int n_split, int n_rows,
+                                               int row0, int row_end, int g, Triple (*sh)[kCombineRows],
+                                               int32_t* __restrict__ out_token, float* __restrict__ out_conf,
+                                               float* __restrict__ out_lse) {
+    const int tx = g & 31, lane = g >> 5;
+    const int row = row0 + tx;
+    Triple x{-INFINITY, 0.f, INT32_MAX};
+    if (row < row_end) {
+        for (int j = lane; j < n_split; j += kCombineLanes) {
+            const size_t o = (size_t)j * n_rows + row;
+            merge_triple(x, pm[o], ps[o], pa[o]);
+        }
+    }
+    sh[lane][tx] = x;
+    __syncthreads();
+    if (lane == 0 && row < row_end) {
+        for (int l = 1; l < kCombineLanes; ++l) {
+            const Triple y = sh[l][tx];
+            if (y.a != INT32_MAX) merge_triple(x, y.m, y.s, y.a);
+        }
+        out_token[row] = x.a;
+        out_conf[row] = 1.0f / x.s;
+        if (out_lse) out_lse[row] = x.m + logf(x.s);
+    }
+    __syncthreads();
+}
+
+}  // namespace psd

@@ -17,6 +17,7 @@
 // Every wait in the kernel is bounded: when a wait runs out the CTA records PSD_ERR_TIMEOUT,
 // raises a CTA-wide abort flag that all roles poll, drains its own asynchronous work with bounded
 // waits, frees its TMEM and returns.
+#include <atomic>
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include "psd_internal.cuh"
@@ -42,6 +43,9 @@ struct TileGeometry {
     int n_vt;        // vocabulary tiles
     int base_units;  // every vocabulary tile has base_units or base_units + 1 units of 16 columns
     int rem;         // the first `rem` vocabulary tiles have base_units + 1
+    int carry;       // 1: a CTA keeps one running triple per row across all its tiles (single row tile)
+                     //    and writes it to split slot blockIdx.x; 0: one triple per (row, vocabulary tile)
+    int band;        // vocabulary tiles per band of the tile order (see decode_tile)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -200,12 +204,19 @@ __device__ __forceinline__ uint64_t l2_policy_evict_normal() {
     return p;
 }
 
-// Tile t -> (row tile, first vocabulary column, width).  Row tiles vary fastest so that the CTAs
-// that run side by side read the same rows of W out of L2.
+// Tile t -> (row tile, first vocabulary column, width).  The vocabulary tiles are grouped in bands
+// of g.band tiles; inside a band the order is (row tile, vocabulary tile) with the vocabulary tile
+// fastest.  The SMs work on consecutive t at any moment, so together they hold one band of W
+// (band * tile bytes, sized to stay in L2 while every row tile passes over it) and a few row tiles of
+// `hidden`, each of which is fetched once per band.
 __device__ __forceinline__ void decode_tile(const TileGeometry& g, int t, int& m_tile, int& v_tile, int& v0,
                                             int& ncols) {
-    m_tile = t % g.n_mt;
-    v_tile = t / g.n_mt;
+    const int per_band = g.band * g.n_mt;
+    const int band = t / per_band;
+    const int r = t - band * per_band;
+    const int width = min(g.band, g.n_vt - band * g.band);   // the last band may be narrower
+    m_tile = r / width;
+    v_tile = band * g.band + (r - m_tile * width);
     const int units0 = v_tile < g.rem ? v_tile * (g.base_units + 1)
                                       : g.rem * (g.base_units + 1) + (v_tile - g.rem) * g.base_units;
     v0 = units0 * 16;
@@ -283,6 +294,13 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+
+    // Programmatic dependent launch: everything above overlapped the tail of the kernel launched
+    // before this one; from here on this kernel reads `hidden` and overwrites the workspace, so it
+    // waits for that kernel to finish.  The kernel launched after this one may start its own
+    // set-up right away (it waits for this grid before touching the partial triples).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -363,6 +381,8 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const int row_in_tile = quarter * 32 + lane;
         int it = 0;
         bool ok = true;
+        float run_m = -INFINITY, run_s = 0.f;
+        int run_a = 0;
         for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
             int m_tile, v_tile, v0, ncols;
             decode_tile(geo, t, m_tile, v_tile, v0, ncols);
@@ -370,8 +390,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, abort_flag, status_dev)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
-            float run_m = -INFINITY, run_s = 0.f;
-            int run_a = 0;
+            if (!geo.carry) { run_m = -INFINITY; run_s = 0.f; run_a = 0; }
             const bool ragged = v0 + ncols > V;      // only the last vocabulary tile can reach past V
             for (int c = 0; c < ncols; c += 32) {
                 float x[32];
@@ -388,9 +407,12 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty_bar[acc]);
+            // A CTA's tiles come in ascending vocabulary order, so a carried triple keeps the lowest
+            // index among equal maxima just as the per-tile triples do after the merge.
+            const bool last_of_cta = t + (int)gridDim.x >= n_tiles;
             const int row = m_tile * BLOCK_M + row_in_tile;
-            if (row < n_rows) {
-                const size_t o = (size_t)v_tile * n_rows + row;
+            if (row < n_rows && (!geo.carry || last_of_cta)) {
+                const size_t o = (size_t)(geo.carry ? (int)blockIdx.x : v_tile) * n_rows + row;
                 pm[o] = run_m;
                 ps[o] = run_s;
                 pa[o] = run_a;
@@ -474,10 +496,24 @@ TileGeometry choose_geometry(int n_rows, int V, int sms, int max_vt) {
     g.n_vt = best_vt;
     g.base_units = units / best_vt;
     g.rem = units % best_vt;
+    g.carry = g.n_mt == 1 ? 1 : 0;
     return g;
 }
 
+std::atomic<int> g_band_bytes{16 << 20};
+
+// Band width: as many vocabulary tiles as fit the L2 budget for W (at least 1, at most all).
+int choose_band(const TileGeometry& g, int H) {
+    const long long tile_bytes = (long long)(g.base_units + (g.rem ? 1 : 0)) * 16 * H * 2;
+    long long b = g_band_bytes.load() / (tile_bytes > 0 ? tile_bytes : 1);
+    if (b < 1) b = 1;
+    if (b > g.n_vt) b = g.n_vt;
+    return (int)b;
+}
+
 }  // namespace
+
+void set_band_bytes(int bytes) { g_band_bytes.store(bytes); }
 
 int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
                          int32_t* status_dev, cudaStream_t st) {
@@ -489,7 +525,8 @@ int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, i
         attr_set = true;
     }
     const int sms = sm_count();
-    const TileGeometry g = choose_geometry(n_rows, V, sms, max_splits(V));
+    TileGeometry g = choose_geometry(n_rows, V, sms, max_splits(V));
+    g.band = choose_band(g, H);
     const int wide_rows = (g.rem ? g.base_units + 1 : g.base_units) * 16;
     const int narrow_rows = g.base_units > 0 ? g.base_units * 16 : wide_rows;
     CUtensorMap map_a, map_bw, map_bn;
@@ -498,10 +535,21 @@ int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, i
         return PSD_ERR_CUDA;
     const int n_tiles = g.n_mt * g.n_vt;
     const int grid = n_tiles < sms ? n_tiles : sms;
-    confidence_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
-                                                                part.s, part.a, status_dev);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
+                                       part.s, part.a, status_dev);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? g.n_vt : PSD_ERR_CUDA;
+    if (e != cudaSuccess) return PSD_ERR_CUDA;
+    return g.carry ? grid : g.n_vt;   // number of split slots written per row
 }
 
 }  // namespace psd

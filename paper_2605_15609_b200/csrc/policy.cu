@@ -3,7 +3,13 @@
 // of int32/fp32 per block, so the kernels are latency bound: every global access is a coalesced
 // row read or write, ranking is done by counting in shared memory, and counts use the block-wide
 // vote instructions.
-#include "psd_internal.cuh"
+//
+// Each stage is a __device__ body that works for any block size >= M (and >= D for acceptance).
+// The bodies take plain (not __restrict__) pointers: in the fused kernel a later stage reads what an
+// earlier stage of the same launch wrote, so no load may go through the read-only data path.
+// The stand-alone kernels wrap one body each, and step_tail_kernel runs the split-V merge and the
+// three bodies back to back for one sequence block, so that a whole step is two launches.
+#include "combine.cuh"
 
 namespace psd {
 namespace {
@@ -36,14 +42,12 @@ __device__ __forceinline__ int node_of(const int32_t* node, int b, int n_nodes) 
     return min(max(nd, 0), n_nodes - 1);
 }
 
-__global__ void select_kernel(const float* __restrict__ conf, const int32_t* __restrict__ tok,
-                              const int32_t* __restrict__ node, int n_nodes,
-                              int32_t* __restrict__ tokens, int32_t* __restrict__ mask, int M,
-                              psd_policy_t p, int32_t* __restrict__ sel, int32_t* __restrict__ n_sel,
-                              int32_t* __restrict__ sel_pos) {
-    extern __shared__ unsigned char smem_raw[];
-    float* s_conf = reinterpret_cast<float*>(smem_raw);
-    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
+__device__ __forceinline__ void select_body(float* s_conf, int* s_flag,
+                                            const float* conf, const int32_t* tok,
+                                            const int32_t* node, int n_nodes,
+                                            int32_t* tokens, int32_t* mask, int M,
+                                            const psd_policy_t& p, int32_t* sel,
+                                            int32_t* n_sel, int32_t* sel_pos) {
     const int b = blockIdx.x, i = threadIdx.x;
     const bool in = i < M;
     const size_t src = ((size_t)b * n_nodes + node_of(node, b, n_nodes)) * M;
@@ -69,14 +73,13 @@ __global__ void select_kernel(const float* __restrict__ conf, const int32_t* __r
     if (i == 0) n_sel[b] = n;
 }
 
-__global__ void build_kernel(const float* __restrict__ conf, const int32_t* __restrict__ tok,
-                             const int32_t* __restrict__ node, int n_nodes,
-                             const int32_t* __restrict__ tokens, const int32_t* __restrict__ mask, int M,
-                             psd_policy_t p, int32_t* __restrict__ sigma, int32_t* __restrict__ n_fill,
-                             int32_t* __restrict__ draft_tokens, int32_t* __restrict__ draft_mask) {
-    extern __shared__ unsigned char smem_raw[];
-    float* s_conf = reinterpret_cast<float*>(smem_raw);
-    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
+__device__ __forceinline__ void build_body(float* s_conf, int* s_flag,
+                                           const float* conf, const int32_t* tok,
+                                           const int32_t* node, int n_nodes,
+                                           const int32_t* tokens, const int32_t* mask,
+                                           int M, const psd_policy_t& p, int32_t* sigma,
+                                           int32_t* n_fill, int32_t* draft_tokens,
+                                           int32_t* draft_mask) {
     const int b = blockIdx.x, i = threadIdx.x, D = p.depth;
     const bool in = i < M;
     const size_t src = ((size_t)b * n_nodes + node_of(node, b, n_nodes)) * M;
@@ -104,18 +107,16 @@ __global__ void build_kernel(const float* __restrict__ conf, const int32_t* __re
     }
 }
 
-__global__ void accept_kernel(const int32_t* __restrict__ tokV, const float* __restrict__ confV,
-                              const int32_t* __restrict__ sigma, const int32_t* __restrict__ n_fill,
-                              const int32_t* __restrict__ draft_tokens, const int32_t* __restrict__ draft_mask,
-                              int M, psd_policy_t p, int32_t* __restrict__ tokens, int32_t* __restrict__ mask,
-                              int32_t* __restrict__ k_star, int32_t* __restrict__ n_spec,
-                              int32_t* __restrict__ n_comm, int32_t* __restrict__ accepted) {
-    extern __shared__ unsigned char smem_raw[];
-    float* s_conf = reinterpret_cast<float*>(smem_raw);
-    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
-    int* s_rank_of = s_flag + blockDim.x;
-    __shared__ int s_nfill[PSD_MAX_DEPTH];
-    __shared__ int s_first_fail;
+__device__ __forceinline__ void accept_body(float* s_conf, int* s_flag, int* s_rank_of, int* s_nfill,
+                                            int* s_first_fail_p,
+                                            const int32_t* tokV, const float* confV,
+                                            const int32_t* sigma, const int32_t* n_fill,
+                                            const int32_t* draft_tokens,
+                                            const int32_t* draft_mask, int M, const psd_policy_t& p,
+                                            int32_t* tokens, int32_t* mask,
+                                            int32_t* k_star, int32_t* n_spec,
+                                            int32_t* n_comm, int32_t* accepted) {
+    int& s_first_fail = *s_first_fail_p;
     const int b = blockIdx.x, i = threadIdx.x, D = p.depth;
     const bool in = i < M;
     const size_t st = (size_t)b * M;
@@ -196,6 +197,102 @@ __global__ void accept_kernel(const int32_t* __restrict__ tokV, const float* __r
     if (accepted && i < D) accepted[(size_t)b * D + i] = i < first_fail ? 1 : 0;
 }
 
+// ---- stand-alone kernels: one body each -----------------------------------------------------
+
+__global__ void select_kernel(const float* __restrict__ conf, const int32_t* __restrict__ tok,
+                              const int32_t* __restrict__ node, int n_nodes,
+                              int32_t* __restrict__ tokens, int32_t* __restrict__ mask, int M,
+                              psd_policy_t p, int32_t* __restrict__ sel, int32_t* __restrict__ n_sel,
+                              int32_t* __restrict__ sel_pos) {
+    extern __shared__ unsigned char smem_raw[];
+    float* s_conf = reinterpret_cast<float*>(smem_raw);
+    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
+    select_body(s_conf, s_flag, conf, tok, node, n_nodes, tokens, mask, M, p, sel, n_sel, sel_pos);
+}
+
+__global__ void build_kernel(const float* __restrict__ conf, const int32_t* __restrict__ tok,
+                             const int32_t* __restrict__ node, int n_nodes,
+                             const int32_t* __restrict__ tokens, const int32_t* __restrict__ mask, int M,
+                             psd_policy_t p, int32_t* __restrict__ sigma, int32_t* __restrict__ n_fill,
+                             int32_t* __restrict__ draft_tokens, int32_t* __restrict__ draft_mask) {
+    extern __shared__ unsigned char smem_raw[];
+    float* s_conf = reinterpret_cast<float*>(smem_raw);
+    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
+    build_body(s_conf, s_flag, conf, tok, node, n_nodes, tokens, mask, M, p, sigma, n_fill, draft_tokens,
+               draft_mask);
+}
+
+__global__ void accept_kernel(const int32_t* __restrict__ tokV, const float* __restrict__ confV,
+                              const int32_t* __restrict__ sigma, const int32_t* __restrict__ n_fill,
+                              const int32_t* __restrict__ draft_tokens, const int32_t* __restrict__ draft_mask,
+                              int M, psd_policy_t p, int32_t* __restrict__ tokens, int32_t* __restrict__ mask,
+                              int32_t* __restrict__ k_star, int32_t* __restrict__ n_spec,
+                              int32_t* __restrict__ n_comm, int32_t* __restrict__ accepted) {
+    extern __shared__ unsigned char smem_raw[];
+    float* s_conf = reinterpret_cast<float*>(smem_raw);
+    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
+    int* s_rank_of = s_flag + blockDim.x;
+    __shared__ int s_nfill[PSD_MAX_DEPTH];
+    __shared__ int s_first_fail;
+    accept_body(s_conf, s_flag, s_rank_of, s_nfill, &s_first_fail, tokV, confV, sigma, n_fill, draft_tokens,
+                draft_mask, M, p, tokens, mask, k_star, n_spec, n_comm, accepted);
+}
+
+// ---- fused tail of a step --------------------------------------------------------------------
+// One thread block per sequence block b: merge the split-V partials of the block's D*M rows
+// (writing tokV / confV), then acceptance on the drafts being verified, the policy on node k*, and
+// the drafts of the next step.  The stages hand data to each other through global memory written
+// and read by the same block, ordered by __syncthreads.
+struct StepTailArgs {
+    const float* pm;
+    const float* ps;
+    const int32_t* pa;
+    int n_split, n_rows, M;
+    psd_policy_t p;
+    int32_t* tokV;
+    float* confV;
+    int32_t *sigma, *n_fill, *draft_tokens, *draft_mask;
+    int32_t *tokens, *mask, *k_star, *n_spec, *n_comm, *sel, *n_sel, *sel_pos;
+};
+
+__global__ void step_tail_kernel(const StepTailArgs a) {
+    extern __shared__ unsigned char smem_raw[];
+    float* s_conf = reinterpret_cast<float*>(smem_raw);
+    int* s_flag = reinterpret_cast<int*>(s_conf + blockDim.x);
+    int* s_rank_of = s_flag + blockDim.x;
+    __shared__ Triple sh[4][kCombineLanes][kCombineRows];
+    __shared__ int s_nfill[PSD_MAX_DEPTH];
+    __shared__ int s_first_fail;
+    const int b = blockIdx.x, D = a.p.depth, M = a.M;
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // the partials come from the kernel launched before
+
+    // split-V merge of rows [b*D*M, (b+1)*D*M): groups of 256 threads take 32 rows at a time
+    const int groups = blockDim.x / kCombineThreads;
+    const int grp = threadIdx.x / kCombineThreads, g = threadIdx.x % kCombineThreads;
+    const int row_begin = b * D * M, row_end = row_begin + D * M;
+    const int n_chunks = (D * M + kCombineRows - 1) / kCombineRows;
+    for (int c0 = 0; c0 < n_chunks; c0 += groups) {
+        const int c = c0 + grp;
+        // threads of a group without a chunk still take part in the barriers inside
+        const int r0 = c < n_chunks ? row_begin + c * kCombineRows : row_end;
+        if (grp < groups)
+            combine_rows32(a.pm, a.ps, a.pa, a.n_split, a.n_rows, r0, row_end, g, sh[grp], a.tokV, a.confV,
+                           nullptr);
+    }
+    __syncthreads();
+
+    accept_body(s_conf, s_flag, s_rank_of, s_nfill, &s_first_fail, a.tokV, a.confV, a.sigma, a.n_fill,
+                a.draft_tokens, a.draft_mask, M, a.p, a.tokens, a.mask, a.k_star, a.n_spec, a.n_comm, nullptr);
+    __syncthreads();
+    select_body(s_conf, s_flag, a.confV, a.tokV, a.k_star, D, a.tokens, a.mask, M, a.p, a.sel, a.n_sel,
+                a.sel_pos);
+    __syncthreads();
+    build_body(s_conf, s_flag, a.confV, a.tokV, a.k_star, D, a.tokens, a.mask, M, a.p, a.sigma, a.n_fill,
+               a.draft_tokens, a.draft_mask);
+}
+
 inline int block_threads(int M) { return ((M + 31) / 32) * 32; }
 
 }  // namespace
@@ -230,6 +327,37 @@ int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma,
                                                 tokens, mask, k_star, n_spec, n_comm, accepted);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
+}
+
+int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_policy_t p,
+                     int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
+                     int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
+                     int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st) {
+    StepTailArgs a;
+    a.pm = part.m; a.ps = part.s; a.pa = part.a;
+    a.n_split = n_split; a.n_rows = n_rows; a.M = M; a.p = p;
+    a.tokV = tokV; a.confV = confV;
+    a.sigma = sigma; a.n_fill = n_fill; a.draft_tokens = draft_tokens; a.draft_mask = draft_mask;
+    a.tokens = tokens; a.mask = mask; a.k_star = k_star; a.n_spec = n_spec; a.n_comm = n_comm;
+    a.sel = sel; a.n_sel = n_sel; a.sel_pos = sel_pos;
+    // a multiple of 256 threads (merge groups), at least one thread per slot and per chain node
+    int need = M > p.depth ? M : p.depth;
+    int t = ((need + kCombineThreads - 1) / kCombineThreads) * kCombineThreads;
+    const int rows_per_block = p.depth * M;
+    while (t < 1024 && t * 2 <= 1024 && rows_per_block > (t / kCombineThreads) * kCombineRows) t *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B);
+    cfg.blockDim = dim3(t);
+    cfg.dynamicSmemBytes = (size_t)t * 12;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, step_tail_kernel, a);
+    count_launch();
+    return e == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }
 
 }  // namespace psd

@@ -59,6 +59,17 @@ int psd_set_confidence_impl(int impl) {
     return g_conf_impl.exchange(impl);
 }
 
+int psd_set_tuning(int knob, int value) {
+    switch (knob) {
+        case PSD_TUNE_BAND_BYTES:
+            if (value < 0) return PSD_ERR_SHAPE;
+            set_band_bytes(value);
+            return PSD_OK;
+        default:
+            return PSD_ERR_UNSUPPORTED;
+    }
+}
+
 int psd_set_kernel_events(void* start_event, void* stop_event) {
     t_ev_start = reinterpret_cast<cudaEvent_t>(start_event);
     t_ev_stop = reinterpret_cast<cudaEvent_t>(stop_event);
@@ -145,18 +156,30 @@ int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V
     const int D = p.depth;
     if ((long long)B * D * M > 2147483647ll) return PSD_ERR_SHAPE;
     const int n_rows = B * D * M;
-    int e = psd_confidence(io->hidden_bf16, io->w_lm_bf16, nullptr, n_rows, H, V, io->tokV, io->confV, nullptr,
-                           workspace, workspace_bytes, status_dev, cuda_stream);
-    if (e) return e;
-    e = psd_verify_accept(io->tokV, io->confV, io->sigma, io->n_fill, io->draft_tokens, io->draft_mask, B, M, p,
-                          io->tokens, io->mask, io->k_star, io->n_spec_accepted, io->n_committed, nullptr,
-                          cuda_stream);
-    if (e) return e;
-    e = psd_select_unmask(io->confV, io->tokV, io->k_star, D, io->tokens, io->mask, B, M, p, io->sel, io->n_sel,
-                          io->sel_pos, cuda_stream);
-    if (e) return e;
-    return psd_build_drafts(io->confV, io->tokV, io->k_star, D, io->tokens, io->mask, B, M, p, io->sigma,
-                            io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream);
+    if (!conf_shape_ok(n_rows, H, V)) return PSD_ERR_SHAPE;
+    if (!workspace) return PSD_ERR_NULL;
+    if (!aligned(io->hidden_bf16, 16) || !aligned(io->w_lm_bf16, 16) || !aligned(workspace, 256) ||
+        !aligned(status_dev, 4))
+        return PSD_ERR_ALIGN;
+    if (workspace_bytes < psd_workspace_bytes(n_rows, H, V)) return PSD_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    Partials part = carve_partials(workspace, n_rows, V);
+    // Two launches: the fused LM-head + confidence kernel, then one kernel per sequence block that
+    // merges the split-V partials and runs acceptance, the policy on node k* and the next drafts.
+    const bool timed = t_ev_start && t_ev_stop;
+    if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
+    int n_split = g_conf_impl.load() == 1
+                      ? launch_confidence_simt(io->hidden_bf16, io->w_lm_bf16, n_rows, H, V, part, st)
+                      : launch_confidence_tc(io->hidden_bf16, io->w_lm_bf16, n_rows, H, V, part, status_dev, st);
+    if (timed) {
+        cudaError_t ce = cudaEventRecord(t_ev_stop, st);
+        t_ev_start = t_ev_stop = nullptr;
+        if (ce != cudaSuccess) return PSD_ERR_CUDA;
+    }
+    if (n_split < 0) return n_split;
+    return launch_step_tail(part, n_split, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
+                            io->draft_tokens, io->draft_mask, io->tokens, io->mask, io->k_star,
+                            io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st);
 }
 
 // Device staging layout of psd_step_host, in order; every piece 256-byte aligned.

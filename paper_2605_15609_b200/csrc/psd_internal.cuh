@@ -39,6 +39,8 @@ int launch_confidence_simt(const void* hidden, const void* w, int n_rows, int H,
 int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V,
                          Partials part, int32_t* status_dev, cudaStream_t st);
 
+void set_band_bytes(int bytes);   // confidence_tc.cu: L2 budget for one band of W in the tile order
+
 // combine.cu: merge n_split partial triples per row.
 int launch_combine(Partials part, int n_split, int n_rows,
                    int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st);
@@ -55,5 +57,11 @@ int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma,
                   const int32_t* draft_tokens, const int32_t* draft_mask, int B, int M, psd_policy_t p,
                   int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec, int32_t* n_comm,
                   int32_t* accepted, cudaStream_t st);
+
+// policy.cu: the whole tail of a step in one launch (split-V merge, acceptance, policy, next drafts).
+int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_policy_t p,
+                     int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
+                     int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
+                     int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st);
 
 }  // namespace psd
