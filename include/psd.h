@@ -270,6 +270,10 @@ int psd_set_confidence_impl(int impl);
  *                        (default 16 MiB); 0 means one vocabulary tile per band
  */
 #define PSD_TUNE_BAND_BYTES 1
+/*   PSD_TUNE_PDL         1 (default): consecutive kernels of a step are launched with programmatic stream
+ *                        serialization, so a kernel's set-up overlaps the end of the one before it;
+ *                        0: plain stream order */
+#define PSD_TUNE_PDL 2
 int psd_set_tuning(int knob, int value);
 
 /*

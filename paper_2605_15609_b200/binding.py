@@ -122,6 +122,7 @@ def psd_set_confidence_impl(impl: int) -> int:
 
 
 PSD_TUNE_BAND_BYTES = 1
+PSD_TUNE_PDL = 2
 
 
 def psd_set_tuning(knob: int, value: int) -> int:

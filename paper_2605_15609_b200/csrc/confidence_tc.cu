@@ -297,10 +297,8 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
     // Programmatic dependent launch: everything above overlapped the tail of the kernel launched
     // before this one; from here on this kernel reads `hidden` and overwrites the workspace, so it
-    // waits for that kernel to finish.  The kernel launched after this one may start its own
-    // set-up right away (it waits for this grid before touching the partial triples).
+    // waits for that kernel to finish.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -422,6 +420,10 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
     tc_fence_before();
     __syncthreads();
+    // This CTA's tiles are done: once every CTA is here the kernel launched next may become resident
+    // and run its set-up (it still waits for this whole grid before it reads the partial triples).
+    // Releasing it any earlier would park its thread blocks on the SMs beside the CTAs still working.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -542,7 +544,10 @@ int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, i
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    // Starting before the kernel ahead has drained hides this kernel's set-up, which matters when the
+    // whole pass takes under 200 us (one row tile).  With many row tiles an early start was measured
+    // to lengthen the pass by 5-8% (8192 rows), so there the kernel keeps plain stream order.
+    attr[0].val.programmaticStreamSerializationAllowed = (pdl_enabled() && g.n_mt == 1) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,

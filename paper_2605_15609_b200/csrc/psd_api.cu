@@ -8,6 +8,7 @@ namespace psd {
 namespace {
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_conf_impl{0};
+std::atomic<int> g_pdl{1};
 thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -28,6 +29,7 @@ bool conf_shape_ok(int n_rows, int H, int V) {
 }  // namespace
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+int pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 }  // namespace psd
 
 using namespace psd;
@@ -64,6 +66,10 @@ int psd_set_tuning(int knob, int value) {
         case PSD_TUNE_BAND_BYTES:
             if (value < 0) return PSD_ERR_SHAPE;
             set_band_bytes(value);
+            return PSD_OK;
+        case PSD_TUNE_PDL:
+            if (value != 0 && value != 1) return PSD_ERR_SHAPE;
+            g_pdl.store(value);
             return PSD_OK;
         default:
             return PSD_ERR_UNSUPPORTED;

@@ -31,6 +31,10 @@ inline Partials carve_partials(void* workspace, int n_rows, int V) {
 
 void count_launch(int n = 1);
 
+// 1 when kernels are launched with programmatic stream serialization (a kernel's set-up overlaps the
+// tail of the one before it), 0 for plain stream order.
+int pdl_enabled();
+
 // confidence_simt.cu: plain CUDA-core kernel. Returns the number of splits written, or < 0.
 int launch_confidence_simt(const void* hidden, const void* w, int n_rows, int H, int V,
                            Partials part, cudaStream_t st);
