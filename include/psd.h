@@ -257,23 +257,30 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
                   void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream);
 
 /*
- * Which kernel psd_confidence uses: 0 = the tcgen05/TMA kernel (default), 1 = a plain
- * CUDA-core kernel kept for cross-checking.  Process-wide; returns the previous value, or
- * PSD_ERR_SHAPE for an unknown value.
+ * Which kernel psd_confidence uses.  Process-wide; returns the previous value, or PSD_ERR_SHAPE for
+ * an unknown value.
+ *   0  (default) and 2: the tcgen05/TMA kernel, one CTA per tile of 128 rows
+ *   1  a plain CUDA-core kernel kept for cross-checking
+ *   3  the tcgen05/TMA kernel that runs pairs of CTAs on tiles of 256 rows (cta_group::2); same
+ *      results up to summation order, measured slower under the board's power cap
  */
 int psd_set_confidence_impl(int impl);
 
 /*
  * Performance knobs (process-wide; results never depend on them).  Returns PSD_OK,
  * PSD_ERR_UNSUPPORTED for an unknown knob or PSD_ERR_SHAPE for a bad value.
- *   PSD_TUNE_BAND_BYTES  bytes of W that one band of the fused kernel's tile order may hold in L2
- *                        (default 16 MiB); 0 means one vocabulary tile per band
+ *   PSD_TUNE_BAND_BYTES  bytes of the operand that one band of the fused kernel's tile order keeps
+ *                        in L2 while the other operand streams past it (default 36 MiB)
  */
 #define PSD_TUNE_BAND_BYTES 1
 /*   PSD_TUNE_PDL         1 (default): consecutive kernels of a step are launched with programmatic stream
  *                        serialization, so a kernel's set-up overlaps the end of the one before it;
  *                        0: plain stream order */
 #define PSD_TUNE_PDL 2
+/*   PSD_TUNE_TILE_ORDER  0 (default): the library picks the tile order with the smaller estimated DRAM
+ *                        traffic; 1: bands of vocabulary tiles (W resident, hidden re-read per band);
+ *                        2: bands of row tiles (hidden resident, W re-read per band) */
+#define PSD_TUNE_TILE_ORDER 3
 int psd_set_tuning(int knob, int value);
 
 /*

@@ -123,6 +123,7 @@ def psd_set_confidence_impl(impl: int) -> int:
 
 PSD_TUNE_BAND_BYTES = 1
 PSD_TUNE_PDL = 2
+PSD_TUNE_TILE_ORDER = 3
 
 
 def psd_set_tuning(knob: int, value: int) -> int:

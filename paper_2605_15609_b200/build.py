@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libpsd_b200.so")
-SOURCES = ["psd_api.cu", "confidence_tc.cu", "confidence_simt.cu", "combine.cu", "policy.cu",
+SOURCES = ["psd_api.cu", "confidence_tc.cu", "confidence_tc2.cu", "confidence_simt.cu", "combine.cu", "policy.cu",
            "confidence_static.cu"]
 EXTRA_SOURCES: list[str] = []
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

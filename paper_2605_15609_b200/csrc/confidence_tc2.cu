@@ -1,0 +1,347 @@
+// Fused LM-head + confidence kernel for sm_100a, CTA-pair version (Sec. 3.1: x^ = argmax_v p(v),
+// c = max_v p(v)).
+//
+// Two CTAs on neighbouring SMs (a cluster of 2) work on one tile of 256 rows x up to 256 vocabulary
+// entries with tcgen05.mma.cta_group::2 (M = 256): each CTA stages its own 128 rows of `hidden` and
+// its own HALF of the W tile, and the tensor cores of both SMs read both halves.  Per 128 x 256 block
+// of logits that is 32 KB per K-slice through L2 and shared memory instead of the single-CTA
+// kernel's 48 KB.  Each CTA keeps the accumulator of its 128 rows in its own TMEM and runs the same
+// epilogue as the single-CTA kernel (thread = row, online max / sum-exp / argmax, one triple per
+// (row, vocabulary tile) to the workspace).  Logits never leave the SM.
+//
+// Measured on B200 at 8192 rows x 126464 x 4096 this version moves a third less data from L2 to the
+// SMs (66 GB against 99 GB per pass) and keeps the tensor pipe as busy (86-88% of cycles), but a
+// pass takes 6.9 ms against the single-CTA kernel's 6.3 ms once the board sits at its power cap
+// (lower SM clocks at the same utilisation).  It is therefore not the default; it is selected with
+// psd_set_confidence_impl(3) and is held to the same parity tests.
+//
+// Roles per CTA: warp 0 = TMA producer (own operands), warp 1 = TMEM allocation, and in the leader
+// CTA (cluster rank 0) the MMA issuer for the pair, warps 2-5 = epilogue.  Barriers:
+//   full[s]      leader only; both CTAs' TMA copies complete their bytes on it
+//   empty[s]     one in each CTA; the leader's tcgen05.commit arrives on both
+//   acc_full[a]  one in each CTA; the leader's tcgen05.commit arrives on both
+//   acc_empty[a] leader only; the 8 epilogue warps of the pair arrive on it
+// No TMA load is multicast.  Every wait is bounded as in the single-CTA kernel; both CTAs meet at a
+// cluster barrier before they free TMEM and exit, so neither touches the other's shared memory after
+// that CTA has gone.
+#include "tc_common.cuh"
+
+namespace psd {
+namespace {
+
+constexpr int STAGES2 = 6;
+constexpr int HALF_N = BLOCK_N / 2;                  // widest half tile of W held by one CTA
+constexpr int B2_BYTES = HALF_N * BLOCK_K * 2;       // 16 KB
+constexpr int STAGE2_BYTES = A_BYTES + B2_BYTES;     // 32 KB
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address, in the cluster's shared window, of the same shared-memory location in CTA `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait on a barrier that threads of the other CTA arrive on.
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                  int32_t* status_dev) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            if (status_dev) atomicCAS(status_dev, 0, (int)PSD_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+// TMA tile load issued by one CTA of a pair into its own shared memory; the bytes are counted on
+// `bar_cluster_addr`, which may be a barrier of the other CTA of the pair.  Not a multicast.
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int x, int y, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y),
+        "l"(policy)
+        : "memory");
+}
+
+// Instruction descriptor, kind::f16, for the pair: D = fp32, A = B = bf16, K-major, M = 256, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_pair(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_f16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                              uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair once every MMA issued
+// so far by this thread has completed.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    const uint16_t both = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(smem_u32(bar)), "h"(both) : "memory");
+}
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b_wide,
+                      const __grid_constant__ CUtensorMap map_b_narrow, TileGeometry geo, int n_rows, int H, int V,
+                      float* __restrict__ pm, float* __restrict__ ps, int32_t* __restrict__ pa,
+                      int32_t* status_dev) {
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment for the 128-byte swizzle; the dynamic shared memory of both CTAs of a cluster
+    // starts at the same offset, so the aligned layouts coincide, as cta_group::2 addressing requires.
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                           ~static_cast<uintptr_t>(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES2 * STAGE2_BYTES);
+    uint64_t* full_bar = bars;                     // [STAGES2] used in the leader
+    uint64_t* empty_bar = bars + STAGES2;          // [STAGES2]
+    uint64_t* acc_full_bar = bars + 2 * STAGES2;   // [2]
+    uint64_t* acc_empty_bar = acc_full_bar + 2;    // [2] used in the leader
+    uint64_t* drain_bar = acc_empty_bar + 2;       // [1] used only when aborting
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain_bar + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int n_tiles = geo.n_mt * geo.n_vt;
+    const int k_blocks = H / BLOCK_K;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES2; ++s) {
+            mbar_init(&full_bar[s], 1);     // the leader's producer arrives (with the byte count of both CTAs)
+            mbar_init(&empty_bar[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&acc_full_bar[a], 1);
+            mbar_init(&acc_empty_bar[a], 8);   // one arrival per epilogue warp of the pair
+        }
+        mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&map_a);
+        tma_prefetch_desc(&map_b_wide);
+        tma_prefetch_desc(&map_b_narrow);
+    }
+    if (warp == 1) {
+        // TMEM for a CTA pair is allocated by one warp of each of the two CTAs.
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync_all();   // barriers of both CTAs are initialised before either CTA signals the other
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (each CTA)
+        if (lane == 0) {
+            // both operands are re-read from L2 many times within a band: mark both to stay (as in the
+            // single-CTA kernel with several row tiles)
+            const uint64_t pol_w = l2_policy_evict_last();
+            const uint64_t pol_h = l2_policy_evict_last();
+            const uint32_t full0 = map_to_cta(smem_u32(&full_bar[0]), 0);   // the leader's full[0]
+            int q = 0;
+            bool ok = true;
+            for (int t = pair_id; t < n_tiles && ok; t += n_pairs) {
+                int m_tile, v_tile, v0, ncols;
+                decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+                const bool wide = v_tile < geo.rem || geo.rem == 0;
+                const CUtensorMap* mb = wide ? &map_b_wide : &map_b_narrow;
+                const int half = ncols >> 1;
+                const uint32_t bytes_pair = 2u * (A_BYTES + (uint32_t)half * BLOCK_K * 2);
+                const int row0 = m_tile * 256 + (int)rank * BLOCK_M;
+                const int col0 = v0 + (int)rank * half;
+                for (int kb = 0; kb < k_blocks; ++kb, ++q) {
+                    const int s = q % STAGES2;
+                    if (!mbar_wait(&empty_bar[s], ((q / STAGES2) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
+                    unsigned char* sa = smem + s * STAGE2_BYTES;
+                    if (leader) mbar_arrive_expect_tx(&full_bar[s], bytes_pair);
+                    const uint32_t fb = full0 + (uint32_t)s * 8;
+                    tma_load_2d_pair(sa, &map_a, fb, kb * BLOCK_K, row0, pol_h);
+                    tma_load_2d_pair(sa + A_BYTES, mb, fb, kb * BLOCK_K, col0, pol_w);
+                }
+            }
+            if (!ok) {
+                // Aborting: no copy may still be in flight when the CTA exits.  The leader can watch its
+                // full barriers (bounded); the other CTA's copies report to the leader's barriers, which
+                // it cannot poll, so it lets a fixed interval pass that is far longer than any copy takes.
+                if (leader) {
+                    const int first = q > STAGES2 ? q - STAGES2 : 0;
+                    for (int i = first; i < q; ++i) {
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait(&full_bar[i % STAGES2], (i / STAGES2) & 1) &&
+                               clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+                    }
+                } else {
+                    const long long t0 = clock64();
+                    while (clock64() - t0 < 2000000ll) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader only)
+        if (leader && lane == 0) {
+            int q = 0, it = 0;
+            bool ok = true;
+            for (int t = pair_id; t < n_tiles && ok; t += n_pairs, ++it) {
+                int m_tile, v_tile, v0, ncols;
+                decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+                const int acc = it & 1;
+                if (!mbar_wait_cluster(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t idesc = umma_idesc_pair(ncols);
+                const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
+                for (int kb = 0; kb < k_blocks; ++kb, ++q) {
+                    const int s = q % STAGES2;
+                    if (!mbar_wait(&full_bar[s], (q / STAGES2) & 1, abort_flag, status_dev)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + s * STAGE2_BYTES);
+                    const uint64_t da = umma_smem_desc(a_addr);
+                    const uint64_t db = umma_smem_desc(a_addr + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_f16_pair(tmem_d, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                    umma_commit_pair(&empty_bar[s]);
+                }
+                if (ok) umma_commit_pair(&acc_full_bar[acc]);
+            }
+            if (!ok) {
+                umma_commit_pair(drain_bar);   // nothing may still be writing TMEM when it is freed
+                const long long t0 = clock64();
+                while (!mbar_try_wait(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5, each CTA)
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t acc_empty0 = map_to_cta(smem_u32(&acc_empty_bar[0]), 0);   // the leader's acc_empty[0]
+        int it = 0;
+        bool ok = true;
+        for (int t = pair_id; t < n_tiles && ok; t += n_pairs, ++it) {
+            int m_tile, v_tile, v0, ncols;
+            decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+            const int acc = it & 1;
+            if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, abort_flag, status_dev)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
+            float run_m = -INFINITY, run_s = 0.f;
+            int run_a = 0;
+            const bool ragged = v0 + ncols > V;
+            for (int c = 0; c < ncols; c += 32) {
+                float x[32];
+                tmem_ld_32x32(taddr + c, x);     // tile widths are multiples of 32 here
+                if (ragged) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (v0 + c + j >= V) x[j] = -INFINITY;
+                }
+                fold_chunk(x, v0 + c, run_m, run_s, run_a);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty0 + (uint32_t)acc * 8);
+            const int row = m_tile * 256 + (int)rank * BLOCK_M + row_in_tile;
+            if (row < n_rows) {
+                const size_t o = (size_t)v_tile * n_rows + row;
+                pm[o] = run_m;
+                ps[o] = run_s;
+                pa[o] = run_a;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncwarp();
+    cluster_sync_all();   // both CTAs are done with each other's shared memory and with TMEM
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace
+
+int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
+                          int32_t* status_dev, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(confidence_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES) !=
+            cudaSuccess)
+            return PSD_ERR_CUDA;
+        attr_set = true;
+    }
+    const int pairs_max = sm_count() / 2;
+    TileGeometry g = choose_geometry(n_rows, V, pairs_max, max_splits(V), 2 * BLOCK_M, 32);
+    choose_order(g, n_rows, H, V, 2 * BLOCK_M, band_bytes(), tile_order());
+    const int wide_half = (g.rem ? g.base_units + 1 : g.base_units) * 16;      // half of unit 32
+    const int narrow_half = g.base_units > 0 ? g.base_units * 16 : wide_half;
+    CUtensorMap map_a, map_bw, map_bn;
+    if (!make_map(&map_a, hidden, n_rows, H, BLOCK_M) || !make_map(&map_bw, w, V, H, wide_half) ||
+        !make_map(&map_bn, w, V, H, narrow_half))
+        return PSD_ERR_CUDA;
+    const int n_tiles = g.n_mt * g.n_vt;
+    const int pairs = n_tiles < pairs_max ? n_tiles : pairs_max;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM2_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 0;   // plain stream order (see the single-CTA launcher)
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc2_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
+                                       part.s, part.a, status_dev);
+    count_launch();
+    if (e != cudaSuccess) return PSD_ERR_CUDA;
+    return g.n_vt;
+}
+
+}  // namespace psd

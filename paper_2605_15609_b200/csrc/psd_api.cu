@@ -9,6 +9,8 @@ namespace {
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_conf_impl{0};
 std::atomic<int> g_pdl{1};
+std::atomic<int> g_band_bytes{36 << 20};
+std::atomic<int> g_tile_order{0};
 thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -30,6 +32,16 @@ bool conf_shape_ok(int n_rows, int H, int V) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 int pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
+long long band_bytes() { return g_band_bytes.load(std::memory_order_relaxed); }
+int tile_order() { return g_tile_order.load(std::memory_order_relaxed); }
+
+int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
+                         int32_t* status_dev, cudaStream_t st) {
+    const int impl = g_conf_impl.load(std::memory_order_relaxed);
+    const bool pairs = impl == 3;   // the single-CTA kernel measured faster at every size (see confidence_tc2.cu)
+    return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, st)
+                 : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, st);
+}
 }  // namespace psd
 
 using namespace psd;
@@ -57,7 +69,7 @@ size_t psd_workspace_bytes(int32_t n_rows, int32_t H, int32_t V) {
 }
 
 int psd_set_confidence_impl(int impl) {
-    if (impl != 0 && impl != 1) return PSD_ERR_SHAPE;
+    if (impl < 0 || impl > 3) return PSD_ERR_SHAPE;
     return g_conf_impl.exchange(impl);
 }
 
@@ -65,7 +77,11 @@ int psd_set_tuning(int knob, int value) {
     switch (knob) {
         case PSD_TUNE_BAND_BYTES:
             if (value < 0) return PSD_ERR_SHAPE;
-            set_band_bytes(value);
+            g_band_bytes.store(value);
+            return PSD_OK;
+        case PSD_TUNE_TILE_ORDER:
+            if (value < 0 || value > 2) return PSD_ERR_SHAPE;
+            g_tile_order.store(value);
             return PSD_OK;
         case PSD_TUNE_PDL:
             if (value != 0 && value != 1) return PSD_ERR_SHAPE;

@@ -39,11 +39,18 @@ int pdl_enabled();
 int launch_confidence_simt(const void* hidden, const void* w, int n_rows, int H, int V,
                            Partials part, cudaStream_t st);
 
-// confidence_tc.cu: tcgen05 + TMA kernel. Returns the number of splits written, or < 0 (psd_status).
+// Tensor-core kernels (tcgen05 + TMA).  Each returns the number of splits written, or < 0 (psd_status).
+// confidence_tc.cu: one CTA per tile of 128 rows; confidence_tc2.cu: a pair of CTAs per tile of 256 rows.
+int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V,
+                          Partials part, int32_t* status_dev, cudaStream_t st);
+int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V,
+                          Partials part, int32_t* status_dev, cudaStream_t st);
+// psd_api.cu: picks the kernel according to psd_set_confidence_impl.
 int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V,
                          Partials part, int32_t* status_dev, cudaStream_t st);
 
-void set_band_bytes(int bytes);   // confidence_tc.cu: L2 budget for one band of W in the tile order
+long long band_bytes();   // psd_api.cu: L2 budget for the operand that a band of the tile order keeps resident
+int tile_order();         // psd_api.cu: 0 = choose, 1 = vocabulary bands, 2 = row bands
 
 // combine.cu: merge n_split partial triples per row.
 int launch_combine(Partials part, int n_split, int n_rows,

@@ -26,7 +26,7 @@ def _rand_inputs(seed, R, H, V, planted=0.5, scale=1.0):
     return gen.bf16_bits(hid), W
 
 
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2, 3])
 def test_tiny_config_all_rows(impl):
     cfg = gen.CONFIGS["tiny"]
     wl = gen.make(cfg)
@@ -46,7 +46,7 @@ RAGGED = [(1, 64, 1), (3, 64, 17), (127, 128, 255), (129, 192, 257), (200, 256, 
 
 
 @pytest.mark.parametrize("R,H,V", RAGGED)
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2, 3])
 def test_ragged_shapes(R, H, V, impl):
     hid, W = _rand_inputs(R * 7 + V, R, H, V)
     tok_o, conf_o, lse_o, gap_o = oracle.confidence(hid, W)
@@ -54,7 +54,7 @@ def test_ragged_shapes(R, H, V, impl):
     check_confidence(tok_g, conf_g, lse_g, tok_o, conf_o, lse_o, gap_o)
 
 
-@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("impl", [0, 1, 2, 3])
 def test_closed_forms_on_gpu(impl):
     # hidden = 0: every logit is 0, so conf = 1/V exactly representable cases and the token is 0.
     H, V = 128, 4096
@@ -87,10 +87,13 @@ def test_two_kernels_agree_and_results_are_deterministic():
     h, w = bf16_dev(hid), bf16_dev(W)
     a = gpu_confidence(h, w, impl=0)
     b = gpu_confidence(h, w, impl=0)
-    c = gpu_confidence(h, w, impl=1)
     for x, y in zip(a, b):
         assert np.array_equal(x, y)                 # bitwise reproducible
-    assert np.array_equal(a[0], c[0]) and np.abs(a[1] - c[1]).max() < 1e-4
+    # CUDA-core kernel, single-CTA tensor-core kernel, CTA-pair tensor-core kernel: the vocabulary is
+    # split differently in each, so sums differ in the last bits but nothing else may
+    for impl in (1, 2, 3):
+        c = gpu_confidence(h, w, impl=impl)
+        assert np.array_equal(a[0], c[0]) and np.abs(a[1] - c[1]).max() < 1e-4
 
 
 def test_nan_inputs_give_nan_confidence_not_a_fault():
