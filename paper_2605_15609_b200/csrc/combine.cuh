@@ -41,7 +41,24 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
     const int row = row0 + tx;
     Triple x{-INFINITY, 0.f, INT32_MAX};
     if (row < row_end) {
-        for (int j = lane; j < n_split; j += kCombineLanes) {
+        // The merge is a dependent chain, the loads are not: fetch a batch of splits first so that their
+        // latencies overlap, then merge them in the same order as a plain loop would.
+        constexpr int kBatch = 8;
+        int j = lane;
+        for (; j + (kBatch - 1) * kCombineLanes < n_split; j += kBatch * kCombineLanes) {
+            float m[kBatch], sv[kBatch];
+            int32_t a[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const size_t o = (size_t)(j + u * kCombineLanes) * n_rows + row;
+                m[u] = pm[o];
+                sv[u] = ps[o];
+                a[u] = pa[o];
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) merge_triple(x, m[u], sv[u], a[u]);
+        }
+        for (; j < n_split; j += kCombineLanes) {
             const size_t o = (size_t)j * n_rows + row;
             merge_triple(x, pm[o], ps[o], pa[o]);
         }
