@@ -374,6 +374,71 @@ def run_ours(args, cfg):
     return 0
 
 
+# ------------------------------------------------------------------------------------ whole loop
+
+def run_loop(args, cfg):
+    """--loop: Algorithm 1 as a whole (psd_decode_blocks) with the table look-up body standing in for
+    the transformer.  Reports time per iteration and the tokens-per-forward-pass of this synthetic
+    body (a property of the toy body, printed as context: the paper's figures come from real models)."""
+    import ctypes
+
+    import torch
+
+    import paper_2605_15609_b200 as psd
+    import psd_inputs as gen
+
+    torch.cuda.set_device(0)
+    B, M, D, H, V = cfg.B, cfg.M, cfg.D, cfg.H, cfg.V
+    W = gen.weights(cfg)
+    table, *_ = gen.table_body(cfg, W)
+    dev = torch.device("cuda", 0)
+    bf = lambda bits: torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    w_dev, t_dev = bf(W), bf(table.reshape(-1, H))
+    hidden = torch.zeros(B * D * M, H, dtype=torch.bfloat16, device=dev)
+    buf = psd.StepBuffers.allocate(B, M, D, H, hidden, w_dev, dev)
+    ws = torch.empty(psd.psd_workspace_bytes(B * D * M, H, V), dtype=torch.uint8, device=dev)
+    scratch = torch.empty(psd.psd_decode_scratch_bytes(B, M), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    passes = torch.zeros(B, dtype=torch.int32, device=dev)
+    pg = psd.policy(tau=float(np.float32(cfg.tau)), k_min=cfg.k_min, k_max=cfg.k_max, depth=D, stride=cfg.stride,
+                    mask_id=cfg.mask_id)
+    user = psd.table_body_user(t_dev.view(B, M, 3, H), B)
+    order = psd.ORDER_ONE_PASS if args.loop == "one_pass" else psd.ORDER_TWO_PASSES
+    stream = torch.cuda.current_stream()
+
+    def decode():
+        buf.tokens.fill_(cfg.mask_id)
+        buf.mask.fill_(1)
+        return psd.psd_decode_blocks(psd.table_body_address(), ctypes.addressof(user), buf, pg, order, 4 * M, scratch,
+                                     ws, status, passes, None, None, stream)
+
+    for _ in range(max(3, min(args.warmup, 5))):
+        decode()
+    n = max(3, min(args.steps, 50))
+    launches0 = psd.psd_launch_count()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    its = fwd = 0
+    for _ in range(n):
+        st = decode()
+        its += st.iterations
+        fwd += st.forward_passes
+    e1.record(stream)
+    torch.cuda.synchronize()
+    secs = e0.elapsed_time(e1) * 1e-3
+    p = passes.cpu().numpy()
+    line = {"metric": "blocks decoded end to end (Algorithm 1 loop, table look-up body)", "value": B * M * n / secs,
+            "unit": "tokens/s", "n_gpus": 1, "steps": n, "ms_per_block_batch": 1e3 * secs / n,
+            "us_per_iteration": 1e6 * secs / max(its, 1), "iterations_per_decode": its / n,
+            "forward_passes_per_decode": fwd / n, "tokens_per_forward_pass_mean": float((M / np.maximum(p, 1)).mean()),
+            "order": args.loop, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": B, "D": D, "M": M, "H": H, "V": V},
+            "gpu_launches": psd.psd_launch_count() - launches0, "status": int(status.item())}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -382,6 +447,9 @@ def main():
     ap.add_argument("--config", default="single_request",
                     help="workload: tiny, single_request, class_7b, batched_serving, deep_sweep[_D1|_D2|_D4]")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--loop", default=None, choices=["one_pass", "two_passes"],
+                    help="time the whole decoding loop (psd_decode_blocks) instead of one step; an extra "
+                         "measurement, not the headline metric")
     ap.add_argument("--profile-only", action="store_true",
                     help="for runs under a profiler: device-resident steps only (no instrumented pass, no "
                          "end-to-end pass, no CPU baseline); the printed line is not a benchmark result")
@@ -396,6 +464,8 @@ def main():
         cfg = gen.CONFIGS[name]
     if args.impl == "reference":
         return run_reference(args, cfg)
+    if args.loop:
+        return run_loop(args, cfg)
     return run_ours(args, cfg)
 
 

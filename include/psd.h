@@ -257,6 +257,79 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
                   void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream);
 
 /*
+ * ---- The whole decoding loop of Algorithm 1 over a batch of blocks ----------------------------------
+ *
+ * The transformer body is the caller's: a function that, given token states on the device, writes
+ * their final hidden states.  n_seq sequences of M slots each: tokens, mask [n_seq, M] int32 (device),
+ * hidden_bf16 [n_seq * M, H] bf16 (device, row (s, i) at s*M + i).  It must enqueue its work on
+ * cuda_stream and return 0, or a negative value that psd_decode_blocks passes on.
+ */
+typedef int (*psd_body_fn)(void* user, const int32_t* tokens, const int32_t* mask, int32_t n_seq, int32_t M,
+                           void* hidden_bf16, void* cuda_stream);
+
+/* Order of operations inside one iteration of psd_decode_blocks. */
+#define PSD_ORDER_TWO_PASSES 0 /* Algorithm 1 as printed: a pass on the state, policy, drafts, a batched
+                                  pass on the D drafts, acceptance                                      */
+#define PSD_ORDER_ONE_PASS 1   /* psd_step: the batched pass on the drafts also serves as the next
+                                  iteration's pass on the state (acceptance, then policy on node k*)   */
+
+typedef struct psd_decode_stats_t {
+    int32_t iterations;     /* iterations of the while loop that ran                                  */
+    int32_t forward_passes; /* calls of the body (batched over all blocks)                            */
+    int32_t masked_left;    /* masked slots left over all blocks: 0 unless max_iterations ran out     */
+} psd_decode_stats_t;
+
+/* Bytes of device scratch psd_decode_blocks needs besides psd_confidence's workspace (0 = bad sizes). */
+size_t psd_decode_scratch_bytes(int32_t B, int32_t M);
+
+/*
+ * psd_decode_blocks — Algorithm 1: repeat { forward pass, policy, drafts, batched verification pass,
+ * hierarchical acceptance } until no block has a masked slot left, or max_iterations.
+ * (Sec. 3.2; Algorithm 1, including its early break when Stage 1 resolves the block.)
+ *
+ * io holds DEVICE pointers.  io->tokens, io->mask [B, M] are the blocks' state, in and out: normally
+ * every slot masked on entry (token = p.mask_id, mask = 1), but any state is accepted.  io->hidden_bf16
+ * is scratch of [B*D*M, H] bf16 that the body fills (the library writes through the pointer although
+ * the field is const).  Every other array of io is scratch/output with the shapes given at
+ * psd_step_io_t; after the call they hold the last iteration's values.  D = p.depth; with D = 1
+ * nothing is speculated and every iteration is one pass (plain parallel decoding).
+ *
+ *   order           PSD_ORDER_TWO_PASSES or PSD_ORDER_ONE_PASS
+ *   scratch         device, 256-byte aligned, >= psd_decode_scratch_bytes(B, M)
+ *   workspace       as for psd_confidence with n_rows = B*D*M
+ *   passes          NULL or device [B] out: forward passes charged to each block (a block is charged
+ *                   for a pass only while it still has masked slots) — M / passes[b] is the block's
+ *                   tokens per forward pass
+ *   done_iteration  NULL or device [B] out: index of the iteration that resolved the block, -1 if none
+ *   trace           NULL or device [max_iterations, B, 4] out: per iteration and block
+ *                   (n_sel, k_star, n_spec_accepted, n_committed); the last three are 0 in iterations
+ *                   that stopped after Stage 1
+ *   stats           host, out
+ * The call is synchronous: after every state update the host reads the number of masked slots (a
+ * 4-byte copy and a stream synchronisation) to decide whether to go on.  It allocates nothing.
+ */
+int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int32_t B, int32_t M, int32_t H,
+                      int32_t V, psd_policy_t p, int32_t order, int32_t max_iterations,
+                      void* scratch, size_t scratch_bytes, void* workspace, size_t workspace_bytes,
+                      int32_t* status_dev, int32_t* passes, int32_t* done_iteration, int32_t* trace,
+                      psd_decode_stats_t* stats, void* cuda_stream);
+
+/*
+ * psd_table_body — a stand-in body for tests and benchmarks (the paper's body is a 7-8B transformer,
+ * which is outside this library): a table look-up with no arithmetic.  user points to a
+ * psd_table_body_t; hidden row (s, i) = table row ((b*M + i)*3 + c), where b = s / (n_seq / B) is the
+ * sequence's block and c in {0, 1, 2} counts the committed neighbours of slot i (slots i-1 and i+1 of
+ * the same sequence with mask 0).  tokens is not read.
+ */
+typedef struct psd_table_body_t {
+    const void* table_bf16; /* [B, M, 3, H] bf16, device, 16-byte aligned */
+    int32_t B;
+    int32_t H;              /* multiple of 8 */
+} psd_table_body_t;
+int psd_table_body(void* user, const int32_t* tokens, const int32_t* mask, int32_t n_seq, int32_t M,
+                   void* hidden_bf16, void* cuda_stream);
+
+/*
  * Which kernel psd_confidence uses.  Process-wide; returns the previous value, or PSD_ERR_SHAPE for
  * an unknown value.
  *   0  (default) and 2: the tcgen05/TMA kernel, one CTA per tile of 128 rows

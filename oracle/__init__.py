@@ -12,6 +12,8 @@ Contents
   build_drafts              Sec. 3.2 Stage 2, Eq. (2); Algorithm 1 "Stage 2"
   verify_accept             Sec. 3.2 Stage 3; Algorithm 1 "Stage 3"
   decode_block              Algorithm 1, the whole loop over one block
+  decode_block_one_pass     the same loop with one model call per iteration (the verification
+                            pass doubles as the next iteration's pass on the state)
 
 Pins: every function above is pinned by ``tests/test_oracle_*.py`` to closed forms,
 brute-force enumeration, library routines and the invariants the paper states.  The parts
@@ -329,5 +331,43 @@ def decode_block(model, M: int, p: Policy, max_steps: int | None = None):
         calls += 1
         tokens, mask, ks, ns, nc, _ = verify_accept(np.asarray(tv)[None], np.asarray(cv)[None],
                                                     sigma, n_fill, dt, dm, p)
+        log.append((int(n_sel[0]), int(ks[0]), int(ns[0]), int(nc[0])))
+    return tokens[0], calls, log
+
+
+def decode_block_one_pass(model, M: int, p: Policy, max_steps: int | None = None):
+    """Algorithm 1 rearranged so that every iteration costs ONE model call.
+
+    The batched pass on the D drafts also scores the root (the current state) and every accepted
+    node, so its predictions for node k* are exactly what Stage 1 of the next iteration would
+    compute on the state that acceptance leaves behind.  An iteration is therefore:
+    model(drafts) -> Stage 3 (acceptance and its extra commit) -> Stage 1 (policy on node k*'s
+    predictions, Eq. (1)) -> Stage 2 (next drafts from the same predictions).  The first iteration
+    verifies D copies of the initial state with nothing speculated.  This is an arrangement of the
+    paper's three stages, not something the paper prints: after the extra commit nothing left exceeds
+    tau, so Stage 1 then adds its k_min fallback positions.
+    Returns the final tokens, the number of model calls, and a per-iteration log of
+    (|T|, k*, n_spec_accepted, n_committed).
+    """
+    p.check()
+    D = p.depth
+    tokens = np.full((1, M), p.mask_id, dtype=np.int32)
+    mask = np.ones((1, M), dtype=np.int32)
+    sigma = np.full((1, M), -1, dtype=np.int32)
+    n_fill = np.zeros((1, D), dtype=np.int32)
+    dt = np.repeat(tokens[:, None, :], D, axis=1)
+    dm = np.repeat(mask[:, None, :], D, axis=1)
+    calls, log = 0, []
+    limit = max_steps if max_steps is not None else 4 * M + 4
+    while mask.any():
+        if len(log) >= limit:
+            raise RuntimeError("decode_block_one_pass did not terminate")
+        tv, cv = model(dt[0], dm[0])
+        calls += 1
+        tv, cv = np.asarray(tv)[None], np.asarray(cv, dtype=np.float64)[None]
+        tokens, mask, ks, ns, nc, _ = verify_accept(tv, cv, sigma, n_fill, dt, dm, p)
+        ck, tk = cv[:, int(ks[0])], tv[:, int(ks[0])]
+        tokens, mask, _, n_sel, _ = select_unmask(ck, tk, tokens, mask, p)
+        sigma, n_fill, dt, dm = build_drafts(ck, tk, tokens, mask, p)
         log.append((int(n_sel[0]), int(ks[0]), int(ns[0]), int(nc[0])))
     return tokens[0], calls, log

@@ -37,6 +37,21 @@ class PsdStepIO(ctypes.Structure):
                                    "n_committed", "sel", "n_sel", "sel_pos")]
 
 
+class PsdDecodeStats(ctypes.Structure):
+    """psd_decode_stats_t"""
+    _fields_ = [("iterations", _i32), ("forward_passes", _i32), ("masked_left", _i32)]
+
+
+class PsdTableBody(ctypes.Structure):
+    """psd_table_body_t"""
+    _fields_ = [("table_bf16", _vp), ("B", _i32), ("H", _i32)]
+
+
+# psd_body_fn
+BODY_FN = ctypes.CFUNCTYPE(ctypes.c_int, _vp, _vp, _vp, _i32, _i32, _vp, _vp)
+ORDER_TWO_PASSES, ORDER_ONE_PASS = 0, 1
+
+
 class PsdError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -70,6 +85,13 @@ def _load() -> ctypes.CDLL:
     lib.psd_step_host_bytes.argtypes = [_i32, _i32, _i32, _i32, _i32]
     lib.psd_step_host.restype = ctypes.c_int
     lib.psd_step_host.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
+    lib.psd_decode_scratch_bytes.restype = _sz
+    lib.psd_decode_scratch_bytes.argtypes = [_i32, _i32]
+    lib.psd_decode_blocks.restype = ctypes.c_int
+    lib.psd_decode_blocks.argtypes = [_vp, _vp, ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _i32, _i32,
+                                      _vp, _sz, _vp, _sz, _vp, _vp, _vp, _vp, ctypes.POINTER(PsdDecodeStats), _vp]
+    lib.psd_table_body.restype = ctypes.c_int
+    lib.psd_table_body.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp]
     lib.psd_set_confidence_impl.restype = ctypes.c_int
     lib.psd_set_confidence_impl.argtypes = [ctypes.c_int]
     lib.psd_set_tuning.restype = ctypes.c_int
@@ -258,3 +280,52 @@ def psd_step_host(buf: StepBuffers, p: PsdPolicy, staging, stream=None) -> int:
                              staging.numel() * staging.element_size(), ctypes.byref(st), _stream(stream)),
            "psd_step_host")
     return int(st.value)
+
+
+def psd_decode_scratch_bytes(B: int, M: int) -> int:
+    return int(LIB.psd_decode_scratch_bytes(B, M))
+
+
+def psd_decode_blocks(body, user, buf: StepBuffers, p: PsdPolicy, order: int, max_iterations: int, scratch,
+                      workspace, status=None, passes=None, done_iteration=None, trace=None, stream=None):
+    """Algorithm 1 over the blocks of ``buf`` (device tensors; ``buf.hidden`` is scratch the body fills).
+
+    ``body`` is either the address of a native ``psd_body_fn`` (an int, e.g. ``table_body_address()``)
+    with ``user`` the address of its argument, or a Python callable
+    ``body(tokens_ptr, mask_ptr, n_seq, M, hidden_ptr, stream_ptr) -> int``.  Returns PsdDecodeStats."""
+    B, M = buf.tokens.shape
+    H = buf.hidden.shape[1]
+    V = buf.w_lm.shape[0]
+    if callable(body):
+        fn = body
+        cb = BODY_FN(lambda u, t, m, n, mm, h, s: int(fn(t, m, n, mm, h, s)))
+        body_ptr = ctypes.cast(cb, _vp)
+    else:
+        cb, body_ptr = None, _vp(int(body))
+    io = buf.io()
+    stats = PsdDecodeStats()
+    code = LIB.psd_decode_blocks(body_ptr, user, ctypes.byref(io), B, M, H, V, p, int(order), int(max_iterations),
+                                 _ptr(scratch), scratch.numel() * scratch.element_size(), _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _ptr(status), _ptr(passes),
+                                 _ptr(done_iteration), _ptr(trace), ctypes.byref(stats), _stream(stream))
+    del cb
+    _check(code, "psd_decode_blocks")
+    return stats
+
+
+def table_body_address() -> int:
+    """Address of the native stand-in body psd_table_body, to pass as ``body``."""
+    return ctypes.cast(LIB.psd_table_body, _vp).value
+
+
+def table_body_user(table, B: int) -> PsdTableBody:
+    """psd_table_body_t for a device table [B, M, 3, H] bf16; keep the object alive during the call and
+    pass ``ctypes.addressof(obj)`` as ``user``."""
+    return PsdTableBody(_ptr(table), int(B), int(table.shape[-1]))
+
+
+def psd_table_body(user: PsdTableBody, mask, hidden, stream=None):
+    """One call of the stand-in body: ``mask`` [n_seq, M] int32 -> ``hidden`` [n_seq*M, H] bf16 (device)."""
+    n_seq, M = mask.shape
+    _check(LIB.psd_table_body(ctypes.addressof(user), None, _ptr(mask), n_seq, M, _ptr(hidden), _stream(stream)),
+           "psd_table_body")

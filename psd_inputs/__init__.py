@@ -189,3 +189,57 @@ def random_state(seed: int, B: int, M: int, V: int, p_masked: float, mask_id: in
             mask[b, i] = 1 if mk else 0
             tokens[b, i] = mask_id if mk else tk
     return tokens, mask
+
+
+# ----------------------------------------------------------------------------------------------
+# A stand-in transformer body for the whole decoding loop: a table of hidden states.
+# ----------------------------------------------------------------------------------------------
+
+TABLE_LEVELS = 3
+
+
+def table_body(cfg: Config, W: np.ndarray, seed: int | None = None):
+    """Hidden states of a toy body whose output depends on the context only through the number of
+    committed neighbours: ``table[b, i, c, :]`` (bf16 bits) is what slot ``i`` of block ``b`` sees when
+    ``c`` of its neighbours ``i-1, i+1`` are committed.  A slot carries a planted peak with probability
+    ``cfg.frac``; its scale starts in [2.75, 3.5] and grows by half a unit (2 nats) per committed
+    neighbour, so that confidences cross the usual thresholds as the block fills, and its token
+    changes from one level to the next with probability ``1 - cfg.rho`` (so that a draft built from an
+    older prediction can be rejected).  Returns (table [B, M, 3, H] uint16, token [B, M, 3] int32,
+    present [B, M] int32, scale [B, M, 3] float64)."""
+    rng = np.random.default_rng(cfg.seed * 7919 + 17 if seed is None else seed)
+    B, M, H, V, L = cfg.B, cfg.M, cfg.H, cfg.V, TABLE_LEVELS
+    present = (rng.random((B, M)) < cfg.frac).astype(np.int32)
+    s0 = rng.uniform(2.75, 3.5, size=(B, M))        # confidence 0.27 .. 0.88 with no committed neighbour
+    scale = s0[:, :, None] + np.arange(L)[None, None, :] * 0.5
+    token = np.empty((B, M, L), dtype=np.int32)
+    token[:, :, 0] = rng.integers(0, V, size=(B, M))
+    for c in range(1, L):
+        keep = rng.random((B, M)) < cfg.rho
+        token[:, :, c] = np.where(keep, token[:, :, c - 1], rng.integers(0, V, size=(B, M)))
+    q = H * W_STD * W_STD
+    table = np.empty((B, M, L, H), dtype=np.uint16)
+    for b in range(B):
+        for i in range(M):
+            for c in range(L):
+                z = rng.standard_normal(H).astype(np.float32)
+                if present[b, i]:
+                    w = bf16_to_f64(W[token[b, i, c]])
+                    g = (np.log(V) + q / 2 + 4.0 * (scale[b, i, c] - 3.0)) / max(float(w @ w), 1e-12)
+                    z = (z.astype(np.float64) + g * w).astype(np.float32)
+                table[b, i, c] = bf16_bits(z)
+    return table, token, present, scale
+
+
+def table_rows(mask: np.ndarray, seq_per_block: int) -> np.ndarray:
+    """Row of the flattened table ``[B*M*3, H]`` that each slot of ``mask[n_seq, M]`` reads:
+    ``((b*M + i)*3 + c)`` with ``b = s // seq_per_block`` and ``c`` = committed neighbours of slot i."""
+    mask = np.asarray(mask)
+    n_seq, M = mask.shape
+    committed = (mask == 0).astype(np.int64)
+    c = np.zeros((n_seq, M), dtype=np.int64)
+    c[:, 1:] += committed[:, :-1]
+    c[:, :-1] += committed[:, 1:]
+    b = (np.arange(n_seq) // seq_per_block)[:, None]
+    i = np.arange(M)[None, :]
+    return (b * M + i) * TABLE_LEVELS + c

@@ -65,3 +65,29 @@ def test_literal_gain_mode_keeps_confidences_low():
     wl = gen.make(cfg)
     _, conf, _, _ = oracle.confidence(wl.hidden_stage1, wl.W)
     assert conf.max() < 0.1
+
+
+def test_table_body_rows_and_levels():
+    """The stand-in body: row indexing by committed neighbours, and confidences that grow with context."""
+    import oracle
+    cfg = gen.Config("t", B=2, H=256, V=1024, M=8, D=2, frac=0.6, s_lo=2.5, s_hi=3.5, seed=3)
+    W = gen.weights(cfg)
+    table, token, present, scale = gen.table_body(cfg, W)
+    assert table.shape == (2, 8, 3, 256) and table.dtype == np.uint16
+    mask = np.array([[1, 1, 0, 1, 0, 0, 1, 1],      # sequence 0 of block 0
+                     [0, 1, 1, 1, 1, 1, 1, 0],      # sequence 1 of block 0
+                     [1, 1, 1, 1, 1, 1, 1, 1],      # block 1
+                     [0, 0, 0, 0, 0, 0, 0, 0]])
+    rows = gen.table_rows(mask, seq_per_block=2)
+    c = rows % 3
+    assert c[0].tolist() == [0, 1, 0, 2, 1, 1, 1, 0]
+    assert c[1].tolist() == [0, 1, 0, 0, 0, 0, 1, 0]
+    assert c[2].tolist() == [0] * 8 and c[3].tolist() == [1, 2, 2, 2, 2, 2, 2, 1]
+    assert (rows // 3 == np.array([[0, 1, 2, 3, 4, 5, 6, 7]] * 2 + [[8, 9, 10, 11, 12, 13, 14, 15]] * 2)).all()
+    tok, conf, _, _ = oracle.confidence(table.reshape(-1, 256), W)
+    tok, conf = tok.reshape(2, 8, 3), conf.reshape(2, 8, 3)
+    pl = present == 1
+    assert pl.any() and (~pl).any()
+    assert (conf[pl][:, 2] > conf[pl][:, 0]).all() and (conf[pl][:, 2] > 0.9).all()
+    assert (tok[pl][:, 2] == token[pl][:, 2]).all()
+    assert (conf[~pl] < 0.1).all()

@@ -374,6 +374,53 @@ def test_loop_always_terminates_within_m_iterations():
         assert sum(n + nc for n, _, _, nc in log) == M      # every slot committed exactly once
 
 
+# ---- the loop with one model call per iteration ------------------------------------------------
+
+def test_one_pass_greedy_collapse_equals_two_pass_greedy():
+    # tau = 1, k = 1, D = 1: nothing exceeds tau, so an iteration is "commit the most confident slot";
+    # both arrangements of Algorithm 1 then make the same calls and reveal the same slots.
+    M = 12
+    p = Policy(tau=1.0, k_min=1, k_max=1, depth=1, mask_id=MASK)
+    a = oracle.decode_block(ToyModel(M), M, p)
+    b = oracle.decode_block_one_pass(ToyModel(M), M, p)
+    assert (a[0] == b[0]).all() and a[1] == b[1] == M
+    assert [n for n, *_ in a[2]] == [n for n, *_ in b[2]] == [1] * M
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 5])
+def test_one_pass_fixed_k_without_threshold_hits(k):
+    # all confidences below tau: the extra commit never fires, each call reveals exactly k slots
+    M = 16
+    p = Policy(tau=1.0, k_min=k, k_max=k, depth=1, mask_id=MASK)
+    tokens, calls, log = oracle.decode_block_one_pass(ToyModel(M), M, p)
+    assert calls == math.ceil(M / k) and (tokens != MASK).all()
+
+
+def test_one_pass_stable_predictions_accept_every_draft():
+    # agreement-only acceptance and predictions that never change: each call accepts the deepest draft
+    # (D-1 speculated slots) and the policy adds one more, so a call reveals D slots; the first call
+    # verifies copies of the empty state and reveals 1.
+    M, D = 17, 4
+    model = ToyModel(M)
+    p = Policy(tau=1.0, k_min=1, k_max=1, depth=D, accept_mode=1, mask_id=MASK)
+    tokens, calls, log = oracle.decode_block_one_pass(model, M, p)
+    assert (tokens == model.target).all()
+    assert log[0] == (1, 0, 0, 0)
+    assert all(ks == D - 1 and ns == D - 1 for _, ks, ns, _ in log[1:-1])
+    assert calls == 1 + math.ceil((M - 1) / D)
+    assert all(K == D for K in model.calls)                # every call is the batched pass over D drafts
+
+
+def test_one_pass_every_slot_committed_once_and_never_more_calls_than_slots():
+    for seed in range(10):
+        M = 24
+        model = ToyModel(M, seed=seed, stable=False)
+        p = Policy(tau=0.8, k_min=1, k_max=6, depth=3, stride=2, mask_id=MASK)
+        tokens, calls, log = oracle.decode_block_one_pass(model, M, p)
+        assert calls == len(log) <= M and (tokens != MASK).all()
+        assert sum(n + nc for n, _, _, nc in log) == M
+
+
 def test_policy_validation():
     for bad in (Policy(k_min=0), Policy(k_min=3, k_max=2), Policy(depth=0), Policy(tau=float("nan")),
                 Policy(accept_mode=5), Policy(stride=-1)):
