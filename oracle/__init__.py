@@ -11,6 +11,7 @@ Contents
   select_unmask             Sec. 3.2 Stage 1, Eq. (1); threshold policy of App. B.2
   build_drafts              Sec. 3.2 Stage 2, Eq. (2); Algorithm 1 "Stage 2"
   verify_accept             Sec. 3.2 Stage 3; Algorithm 1 "Stage 3"
+  build_drafts_dag, verify_accept_dag   the same two stages for a general multi-parent draft graph
   decode_block              Algorithm 1, the whole loop over one block
   decode_block_one_pass     the same loop with one model call per iteration (the verification
                             pass doubles as the next iteration's pass on the state)
@@ -371,3 +372,123 @@ def decode_block_one_pass(model, M: int, p: Policy, max_steps: int | None = None
         sigma, n_fill, dt, dm = build_drafts(ck, tk, tokens, mask, p)
         log.append((int(n_sel[0]), int(ks[0]), int(ns[0]), int(nc[0])))
     return tokens[0], calls, log
+
+
+# --------------------------------------------------------------------------------------
+# General draft graph (Sec. 3.2 Stage 2-3; Algorithm 1 with a DAG): nodes are sets of RANKS of
+# the speculative ordering sigma; an edge (p, k) exists whenever S_p is a strict subset of S_k.
+# --------------------------------------------------------------------------------------
+
+def dag_edges(node_ranks):
+    """All (p, k) with S_p a strict subset of S_k (Sec. 3.2: "an edge exists whenever S_p ⊂ S_k")."""
+    sets = [frozenset(s) for s in node_ranks]
+    return [(p, k) for k in range(len(sets)) for p in range(len(sets)) if sets[p] < sets[k]]
+
+
+def build_drafts_dag(conf, tok, tokens, mask, p: Policy, node_ranks):
+    """Stage 2 for a draft graph.  node_ranks[k] = the ranks j (0-based positions in sigma) that node k
+    speculates; node 0 must be the root (empty).  With m residual slots only ranks < m exist:
+    S_k = {sigma_j : j in node_ranks[k], j < m}; draft k is Eq. (2).
+    Returns sigma[B, M], n_fill[B, K] (= |S_k|), draft_tokens[B, K, M], draft_mask[B, K, M]."""
+    p.check()
+    if len(node_ranks) < 1 or len(node_ranks[0]) != 0:
+        raise ValueError("node 0 must be the root (no speculated ranks)")
+    conf = np.asarray(conf, dtype=np.float64)
+    tok = np.asarray(tok)
+    tokens = np.asarray(tokens, dtype=np.int32)
+    mask = np.asarray(mask, dtype=np.int32)
+    B, M = mask.shape
+    K = len(node_ranks)
+    sigma = np.full((B, M), -1, dtype=np.int32)
+    n_fill = np.zeros((B, K), dtype=np.int32)
+    draft_tokens = np.empty((B, K, M), dtype=np.int32)
+    draft_mask = np.empty((B, K, M), dtype=np.int32)
+    for b in range(B):
+        residual = [i for i in range(M) if mask[b, i] != 0]
+        order = sorted(residual, key=lambda i: _rank_key(conf[b], i))
+        m = len(order)
+        sigma[b, :m] = order
+        for k in range(K):
+            S = [order[j] for j in sorted(node_ranks[k]) if j < m]
+            n_fill[b, k] = len(S)
+            draft_tokens[b, k] = tokens[b]
+            draft_mask[b, k] = mask[b]
+            for i in S:                              # Eq. (2)
+                draft_tokens[b, k, i] = tok[b, i]
+                draft_mask[b, k, i] = 0
+    return sigma, n_fill, draft_tokens, draft_mask
+
+
+def verify_accept_dag(tokV, confV, sigma, draft_tokens, draft_mask, p: Policy, node_ranks, edges=None):
+    """Stage 3 for a draft graph (Algorithm 1 "Stage 3").  `edges` = list of (p, k) with S_p a strict
+    subset of S_k; None means every such pair (the paper's definition of the edge set).
+
+    The root is accepted.  Nodes are visited in topological order (fewer speculated ranks first, lower
+    index first among equals); node k is accepted iff some ACCEPTED p with an edge (p, k) passes
+    A_pi(x~_{k,i}, x^_{p,i}, c_{p,i}) on every i in S_k \\ S_p (an empty difference passes).
+    k* = the accepted node with the largest |S_k|, lowest index among equals; then the state becomes
+    draft k* and node k*'s own predictions above tau are committed as well.
+    Returns tokens, mask, k_star[B], n_spec_accepted[B], n_committed[B], accepted[B, K]."""
+    p.check()
+    tokV = np.asarray(tokV)
+    confV = np.asarray(confV, dtype=np.float64)
+    B, K, M = draft_tokens.shape
+    if edges is None:
+        edges = dag_edges(node_ranks)
+    for (q, k) in edges:
+        if not frozenset(node_ranks[q]) < frozenset(node_ranks[k]):
+            raise ValueError("an edge (p, k) needs S_p to be a strict subset of S_k")
+    topo = sorted(range(K), key=lambda k: (len(node_ranks[k]), k))
+    tokens = np.empty((B, M), dtype=np.int32)
+    mask = np.empty((B, M), dtype=np.int32)
+    k_star = np.zeros(B, dtype=np.int32)
+    n_spec = np.zeros(B, dtype=np.int32)
+    n_comm = np.zeros(B, dtype=np.int32)
+    accepted = np.zeros((B, K), dtype=np.int32)
+    for b in range(B):
+        m = int((sigma[b] >= 0).sum())
+        S = [set(int(sigma[b, j]) for j in node_ranks[k] if j < m) for k in range(K)]
+        pol = {}
+        accepted[b, 0] = 1
+        for k in topo:
+            if k == 0:
+                continue
+            for (q, kk) in edges:
+                if kk != k or not accepted[b, q]:
+                    continue
+                ok = True
+                for i in S[k] - S[q]:
+                    agree = int(tokV[b, q, i]) == int(draft_tokens[b, k, i])
+                    if p.accept_mode == ACCEPT_AGREE_AND_CONF:
+                        good = agree and float(confV[b, q, i]) > p.tau
+                    elif p.accept_mode == ACCEPT_AGREE_ONLY:
+                        good = agree
+                    else:
+                        if q not in pol:
+                            pol[q] = set(policy_set(confV[b, q], draft_mask[b, q], p))
+                        good = agree and i in pol[q]
+                    ok = ok and good
+                if ok:
+                    accepted[b, k] = 1
+                    break
+        best, best_n = 0, -1
+        for k in range(K):
+            if accepted[b, k] and len(S[k]) > best_n:
+                best, best_n = k, len(S[k])
+        k_star[b] = best
+        n_spec[b] = best_n
+        tokens[b] = draft_tokens[b, best]
+        mask[b] = draft_mask[b, best]
+        extra = 0
+        for i in range(M):
+            if mask[b, i] != 0 and float(confV[b, best, i]) > p.tau:
+                tokens[b, i] = tokV[b, best, i]
+                mask[b, i] = 0
+                extra += 1
+        n_comm[b] = best_n + extra
+    return tokens, mask, k_star, n_spec, n_comm, accepted
+
+
+def chain_as_dag(depth: int, step: int):
+    """The chain of `depth` nodes (root included) adding `step` ranks per depth, as node rank sets."""
+    return [set(range(d * step)) for d in range(depth)]
