@@ -257,6 +257,58 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
                   void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream);
 
 /*
+ * ---- General draft graph (multi-parent DAG) ------------------------------------------------------------
+ * (Sec. 3.2 Stage 2: nodes k with subsets S_k of {sigma_1..sigma_m}, an edge (p, k) whenever S_p is a
+ *  strict subset of S_k, a node may have several parents; Algorithm 1 Stage 3 for the acceptance.)
+ *
+ * The graph is fixed at inference time and expressed over RANKS of the speculative ordering: bit j of
+ * ranks[k] set means that node k speculates sigma_{j+1} (the slot with the (j+1)-th highest cached
+ * confidence among the residual masked slots).  Only the 64 best ranks can be speculated.  Node 0 is
+ * the root (ranks[0] = 0).  When fewer than 64 residual slots exist, ranks beyond them drop out of
+ * every node.  bit p of parents[k] set means that (p, k) is an edge; S_p must be a strict subset of
+ * S_k.  The chain of psd_build_drafts is the special case ranks[d] = lowest d*stride bits,
+ * parents[d] = {d-1}.
+ */
+#define PSD_MAX_DAG_NODES 64
+typedef struct psd_dag_t {
+    int32_t n_nodes;                      /* K, 1 .. PSD_MAX_DAG_NODES */
+    int32_t reserved;
+    uint64_t ranks[PSD_MAX_DAG_NODES];
+    uint64_t parents[PSD_MAX_DAG_NODES];
+} psd_dag_t;
+
+/*
+ * Fills *g (host memory) from n_nodes rank words and, optionally, parent words.  parents == NULL makes
+ * every strict-subset pair an edge (the paper's edge set).  Returns PSD_ERR_SHAPE if node 0 is not the
+ * root, n_nodes is out of range, or an edge is not between a strict subset and its superset.
+ */
+int psd_dag_init(psd_dag_t* g, int32_t n_nodes, const uint64_t* ranks, const uint64_t* parents);
+
+/*
+ * psd_build_drafts_dag — psd_build_drafts for a draft graph: sigma as there; node k fills
+ * S_k = {sigma_{j+1} : bit j of g->ranks[k], j < m}; Eq. (2).  g is a HOST pointer.
+ *   n_fill [B, K] out: |S_k|;  draft_tokens, draft_mask [B, K, M] out.  p is not used (kept for symmetry).
+ */
+int psd_build_drafts_dag(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
+                         const int32_t* tokens, const int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
+                         const psd_dag_t* g, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
+                         int32_t* draft_mask, void* cuda_stream);
+
+/*
+ * psd_verify_accept_dag — hierarchical acceptance over the graph, then the commit (Algorithm 1 Stage 3).
+ * tokV, confV [B, K, M] are psd_confidence's outputs on the K drafts.  The root is accepted; in
+ * topological order (fewer speculated ranks first, lower index among equals) node k is accepted iff
+ * some accepted parent p passes A_pi(x~_{k,i}, x^_{p,i}, c_{p,i}) (p.accept_mode) on every slot of
+ * S_k \ S_p; an empty difference passes.  k* = the accepted node with the largest |S_k|, lowest index
+ * among equals.  Then as psd_verify_accept: tokens, mask <- draft k*, plus node k*'s own predictions
+ * above tau.  accepted [B, K] out or NULL.  p.depth and p.stride are not used.
+ */
+int psd_verify_accept_dag(const int32_t* tokV, const float* confV, const int32_t* sigma,
+                          const int32_t* draft_tokens, const int32_t* draft_mask, int32_t B, int32_t M,
+                          psd_policy_t p, const psd_dag_t* g, int32_t* tokens, int32_t* mask, int32_t* k_star,
+                          int32_t* n_spec_accepted, int32_t* n_committed, int32_t* accepted, void* cuda_stream);
+
+/*
  * ---- The whole decoding loop of Algorithm 1 over a batch of blocks ----------------------------------
  *
  * The transformer body is the caller's: a function that, given token states on the device, writes

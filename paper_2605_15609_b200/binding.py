@@ -37,6 +37,12 @@ class PsdStepIO(ctypes.Structure):
                                    "n_committed", "sel", "n_sel", "sel_pos")]
 
 
+class PsdDag(ctypes.Structure):
+    """psd_dag_t"""
+    _fields_ = [("n_nodes", _i32), ("reserved", _i32), ("ranks", ctypes.c_uint64 * 64),
+                ("parents", ctypes.c_uint64 * 64)]
+
+
 class PsdDecodeStats(ctypes.Structure):
     """psd_decode_stats_t"""
     _fields_ = [("iterations", _i32), ("forward_passes", _i32), ("masked_left", _i32)]
@@ -85,6 +91,14 @@ def _load() -> ctypes.CDLL:
     lib.psd_step_host_bytes.argtypes = [_i32, _i32, _i32, _i32, _i32]
     lib.psd_step_host.restype = ctypes.c_int
     lib.psd_step_host.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
+    lib.psd_dag_init.restype = ctypes.c_int
+    lib.psd_dag_init.argtypes = [ctypes.POINTER(PsdDag), _i32, _vp, _vp]
+    lib.psd_build_drafts_dag.restype = ctypes.c_int
+    lib.psd_build_drafts_dag.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _i32, _i32, pol, ctypes.POINTER(PsdDag), _vp,
+                                         _vp, _vp, _vp, _vp]
+    lib.psd_verify_accept_dag.restype = ctypes.c_int
+    lib.psd_verify_accept_dag.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i32, pol, ctypes.POINTER(PsdDag), _vp, _vp,
+                                          _vp, _vp, _vp, _vp, _vp]
     lib.psd_decode_scratch_bytes.restype = _sz
     lib.psd_decode_scratch_bytes.argtypes = [_i32, _i32]
     lib.psd_decode_blocks.restype = ctypes.c_int
@@ -329,3 +343,36 @@ def psd_table_body(user: PsdTableBody, mask, hidden, stream=None):
     n_seq, M = mask.shape
     _check(LIB.psd_table_body(ctypes.addressof(user), None, _ptr(mask), n_seq, M, _ptr(hidden), _stream(stream)),
            "psd_table_body")
+
+
+def psd_dag_init(node_ranks, edges=None) -> PsdDag:
+    """A draft graph from node rank sets (node 0 = the root, empty) and, optionally, an edge list
+    [(p, k), ...]; without one every strict-subset pair is an edge."""
+    K = len(node_ranks)
+    ranks = (ctypes.c_uint64 * max(K, 1))(*[sum(1 << int(j) for j in s) for s in node_ranks])
+    par = None
+    if edges is not None:
+        words = [0] * K
+        for q, k in edges:
+            words[k] |= 1 << q
+        par = (ctypes.c_uint64 * max(K, 1))(*words)
+    g = PsdDag()
+    _check(LIB.psd_dag_init(ctypes.byref(g), K, ctypes.cast(ranks, _vp), ctypes.cast(par, _vp) if par else None),
+           "psd_dag_init")
+    return g
+
+
+def psd_build_drafts_dag(conf, tok, tokens, mask, p: PsdPolicy, g: PsdDag, sigma, n_fill, draft_tokens, draft_mask,
+                         node=None, n_nodes=1, stream=None):
+    B, M = mask.shape
+    _check(LIB.psd_build_drafts_dag(_ptr(conf), _ptr(tok), _ptr(node), n_nodes, _ptr(tokens), _ptr(mask), B, M, p,
+                                    ctypes.byref(g), _ptr(sigma), _ptr(n_fill), _ptr(draft_tokens), _ptr(draft_mask),
+                                    _stream(stream)), "psd_build_drafts_dag")
+
+
+def psd_verify_accept_dag(tokV, confV, sigma, draft_tokens, draft_mask, p: PsdPolicy, g: PsdDag, tokens, mask, k_star,
+                          n_spec_accepted, n_committed, accepted=None, stream=None):
+    B, M = tokens.shape
+    _check(LIB.psd_verify_accept_dag(_ptr(tokV), _ptr(confV), _ptr(sigma), _ptr(draft_tokens), _ptr(draft_mask), B, M,
+                                     p, ctypes.byref(g), _ptr(tokens), _ptr(mask), _ptr(k_star), _ptr(n_spec_accepted),
+                                     _ptr(n_committed), _ptr(accepted), _stream(stream)), "psd_verify_accept_dag")
