@@ -396,7 +396,8 @@ def run_loop(args, cfg):
     w_dev, t_dev = bf(W), bf(table.reshape(-1, H))
     hidden = torch.zeros(B * D * M, H, dtype=torch.bfloat16, device=dev)
     buf = psd.StepBuffers.allocate(B, M, D, H, hidden, w_dev, dev)
-    ws = torch.empty(psd.psd_workspace_bytes(B * D * M, H, V), dtype=torch.uint8, device=dev)
+    ws = torch.empty(psd.psd_compact_workspace_bytes(B * D * M, H, V), dtype=torch.uint8, device=dev)
+    psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, 1 if args.compact else 0)
     scratch = torch.empty(psd.psd_decode_scratch_bytes(B, M), dtype=torch.uint8, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     passes = torch.zeros(B, dtype=torch.int32, device=dev)
@@ -432,7 +433,7 @@ def run_loop(args, cfg):
             "unit": "tokens/s", "n_gpus": 1, "steps": n, "ms_per_block_batch": 1e3 * secs / n,
             "us_per_iteration": 1e6 * secs / max(its, 1), "iterations_per_decode": its / n,
             "forward_passes_per_decode": fwd / n, "tokens_per_forward_pass_mean": float((M / np.maximum(p, 1)).mean()),
-            "order": args.loop, "dtype": "bf16", "data": "synthetic",
+            "order": args.loop, "compact_rows": bool(args.compact), "dtype": "bf16", "data": "synthetic",
             "config": {"workload": cfg.name, "B": B, "D": D, "M": M, "H": H, "V": V},
             "gpu_launches": psd.psd_launch_count() - launches0, "status": int(status.item())}
     print(json.dumps(line), flush=True)
@@ -450,6 +451,8 @@ def main():
     ap.add_argument("--loop", default=None, choices=["one_pass", "two_passes"],
                     help="time the whole decoding loop (psd_decode_blocks) instead of one step; an extra "
                          "measurement, not the headline metric")
+    ap.add_argument("--compact", action="store_true",
+                    help="with --loop one_pass: score only the rows of slots still masked in their draft")
     ap.add_argument("--profile-only", action="store_true",
                     help="for runs under a profiler: device-resident steps only (no instrumented pass, no "
                          "end-to-end pass, no CPU baseline); the printed line is not a benchmark result")

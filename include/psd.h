@@ -86,6 +86,13 @@ const char* psd_status_string(int code);
 size_t psd_workspace_bytes(int32_t n_rows, int32_t H, int32_t V);
 
 /*
+ * Bytes of scratch for the paths that first copy the rows to score into a dense buffer: psd_confidence
+ * with a row list, and psd_step / psd_decode_blocks with PSD_TUNE_COMPACT_ROWS on (n_rows = B*D*M).
+ * Always >= psd_workspace_bytes.  Returns 0 for invalid sizes.
+ */
+size_t psd_compact_workspace_bytes(int32_t n_rows, int32_t H, int32_t V);
+
+/*
  * psd_confidence — LM head + softmax max-probability + argmax, without ever storing logits.
  * (Sec. 3.1: x^_i and c_i; used for the single sequence of Stage 1 and for all drafts of the
  *  batched verification pass of Stage 3.)
@@ -97,7 +104,9 @@ size_t psd_workspace_bytes(int32_t n_rows, int32_t H, int32_t V);
  *
  *   hidden_bf16  [n_rows, H] bf16, 16-byte aligned, device
  *   w_lm_bf16    [V, H]      bf16, 16-byte aligned, device
- *   row_ids      reserved for a gather list of active rows; must be NULL
+ *   row_ids      NULL, or a device list [n_rows] int32 of the rows of hidden_bf16 to score (a gather list:
+ *                output r belongs to hidden row row_ids[r]; hidden_bf16 may then have any number of rows).
+ *                The workspace must then hold psd_compact_workspace_bytes(n_rows, H, V)
  *   n_rows >= 1;  H >= 64 and a multiple of 64;  1 <= V < 2^31 - 256
  *   out_token    [n_rows] int32;  out_conf [n_rows] fp32;  out_lse [n_rows] fp32 or NULL
  *   workspace    >= psd_workspace_bytes(n_rows, H, V) bytes, 256-byte aligned, device; contents
@@ -406,6 +415,12 @@ int psd_set_confidence_impl(int impl);
  *                        traffic; 1: bands of vocabulary tiles (W resident, hidden re-read per band);
  *                        2: bands of row tiles (hidden resident, W re-read per band) */
 #define PSD_TUNE_TILE_ORDER 3
+/*   PSD_TUNE_COMPACT_ROWS  psd_step scores only the rows of slots that are still masked in their draft
+ *                        (Sec. 3.2 Stage 3: "each masked position"): 0 (default) off; 1 on when the
+ *                        batch has more than 128 rows; 2 always.  With it on, the workspace must hold
+ *                        psd_compact_workspace_bytes, and entries of tokV / confV that belong to
+ *                        committed slots are left as they were (no stage reads them) */
+#define PSD_TUNE_COMPACT_ROWS 4
 int psd_set_tuning(int knob, int value);
 
 /*

@@ -74,6 +74,8 @@ def _load() -> ctypes.CDLL:
     lib.psd_status_string.argtypes = [ctypes.c_int]
     lib.psd_workspace_bytes.restype = _sz
     lib.psd_workspace_bytes.argtypes = [_i32, _i32, _i32]
+    lib.psd_compact_workspace_bytes.restype = _sz
+    lib.psd_compact_workspace_bytes.argtypes = [_i32, _i32, _i32]
     lib.psd_confidence.restype = ctypes.c_int
     lib.psd_confidence.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
     lib.psd_confidence_static.restype = ctypes.c_int
@@ -153,6 +155,10 @@ def psd_workspace_bytes(n_rows: int, H: int, V: int) -> int:
     return int(LIB.psd_workspace_bytes(n_rows, H, V))
 
 
+def psd_compact_workspace_bytes(n_rows: int, H: int, V: int) -> int:
+    return int(LIB.psd_compact_workspace_bytes(n_rows, H, V))
+
+
 def psd_set_confidence_impl(impl: int) -> int:
     return int(LIB.psd_set_confidence_impl(int(impl)))
 
@@ -160,6 +166,7 @@ def psd_set_confidence_impl(impl: int) -> int:
 PSD_TUNE_BAND_BYTES = 1
 PSD_TUNE_PDL = 2
 PSD_TUNE_TILE_ORDER = 3
+PSD_TUNE_COMPACT_ROWS = 4
 
 
 def psd_set_tuning(knob: int, value: int) -> int:
@@ -183,6 +190,8 @@ def psd_confidence(hidden, w_lm, out_token, out_conf, out_lse=None, workspace=No
                    row_ids=None):
     """hidden [n_rows, H] bf16, w_lm [V, H] bf16 -> out_token int32, out_conf fp32 (and out_lse) [n_rows]."""
     n_rows, H = hidden.shape
+    if row_ids is not None:
+        n_rows = row_ids.numel()
     V = w_lm.shape[0]
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(LIB.psd_confidence(_ptr(hidden), _ptr(w_lm), _ptr(row_ids), n_rows, H, V, _ptr(out_token),

@@ -36,11 +36,13 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
                                                const int32_t* __restrict__ pa, int n_split, int n_rows,
                                                int row0, int row_end, int g, Triple (*sh)[kCombineRows],
                                                int32_t* __restrict__ out_token, float* __restrict__ out_conf,
-                                               float* __restrict__ out_lse) {
+                                               float* __restrict__ out_lse, const int32_t* __restrict__ pos = nullptr) {
     const int tx = g & 31, lane = g >> 5;
-    const int row = row0 + tx;
+    const int out_row = row0 + tx;
+    // with compacted rows the partials of output row r sit in column pos[r]; -1 = the row was not scored
+    const int row = out_row < row_end ? (pos ? pos[out_row] : out_row) : -1;
     Triple x{-INFINITY, 0.f, INT32_MAX};
-    if (row < row_end) {
+    if (row >= 0) {
         // The merge is a dependent chain, the loads are not: fetch a batch of splits first so that their
         // latencies overlap, then merge them in the same order as a plain loop would.
         constexpr int kBatch = 8;
@@ -65,14 +67,14 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
     }
     sh[lane][tx] = x;
     __syncthreads();
-    if (lane == 0 && row < row_end) {
+    if (lane == 0 && row >= 0) {
         for (int l = 1; l < kCombineLanes; ++l) {
             const Triple y = sh[l][tx];
             if (y.a != INT32_MAX) merge_triple(x, y.m, y.s, y.a);
         }
-        out_token[row] = x.a;
-        out_conf[row] = 1.0f / x.s;
-        if (out_lse) out_lse[row] = x.m + logf(x.s);
+        out_token[out_row] = x.a;
+        out_conf[out_row] = 1.0f / x.s;
+        if (out_lse) out_lse[out_row] = x.m + logf(x.s);
     }
     __syncthreads();
 }

@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b_wide,
                      const __grid_constant__ CUtensorMap map_b_narrow, TileGeometry geo, int n_rows, int H, int V,
                      float* __restrict__ pm, float* __restrict__ ps, int32_t* __restrict__ pa,
-                     int32_t* status_dev) {
+                     int32_t* status_dev, const int32_t* __restrict__ n_rows_dev) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: required by the 128-byte swizzle pattern shared by TMA and the MMA descriptors
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -42,7 +42,6 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_tiles = geo.n_mt * geo.n_vt;
     const int k_blocks = H / BLOCK_K;
 
     if (threadIdx.x == 0) {
@@ -77,6 +76,16 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     // before this one; from here on this kernel reads `hidden` and overwrites the workspace, so it
     // waits for that kernel to finish.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // The number of rows to score may be known only on the device (rows compacted by the kernel
+    // ahead): n_rows then stays the capacity (tensor map, stride of the partial arrays) and the tile
+    // list shrinks to the row tiles that hold rows.
+    int n_rows_act = n_rows;
+    if (n_rows_dev) {
+        n_rows_act = min(max(*n_rows_dev, 0), n_rows);
+        geo.n_mt = (n_rows_act + BLOCK_M - 1) / BLOCK_M;
+    }
+    const int n_tiles = geo.n_mt * geo.n_vt;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -191,7 +200,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             // index among equal maxima just as the per-tile triples do after the merge.
             const bool last_of_cta = t + (int)gridDim.x >= n_tiles;
             const int row = m_tile * BLOCK_M + row_in_tile;
-            if (row < n_rows && (!geo.carry || last_of_cta)) {
+            if (row < n_rows_act && (!geo.carry || last_of_cta)) {
                 const size_t o = (size_t)(geo.carry ? (int)blockIdx.x : v_tile) * n_rows + row;
                 pm[o] = run_m;
                 ps[o] = run_s;
@@ -216,7 +225,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 }  // namespace
 
 int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
-                          int32_t* status_dev, cudaStream_t st) {
+                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(confidence_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) !=
@@ -250,7 +259,7 @@ int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
-                                       part.s, part.a, status_dev);
+                                       part.s, part.a, status_dev, n_rows_dev);
     count_launch();
     if (e != cudaSuccess) return PSD_ERR_CUDA;
     return g.carry ? grid : g.n_vt;   // number of split slots written per row

@@ -122,7 +122,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b_wide,
                       const __grid_constant__ CUtensorMap map_b_narrow, TileGeometry geo, int n_rows, int H, int V,
                       float* __restrict__ pm, float* __restrict__ ps, int32_t* __restrict__ pa,
-                      int32_t* status_dev) {
+                      int32_t* status_dev, const int32_t* __restrict__ n_rows_dev) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the 128-byte swizzle; the dynamic shared memory of both CTAs of a cluster
     // starts at the same offset, so the aligned layouts coincide, as cta_group::2 addressing requires.
@@ -141,7 +141,6 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
     const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int n_tiles = geo.n_mt * geo.n_vt;
     const int k_blocks = H / BLOCK_K;
 
     if (threadIdx.x == 0) {
@@ -175,6 +174,14 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     const uint32_t tmem_base = *tmem_holder;
 
     asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // rows known only on the device (see the single-CTA kernel): the tile list shrinks accordingly
+    int n_rows_act = n_rows;
+    if (n_rows_dev) {
+        n_rows_act = min(max(*n_rows_dev, 0), n_rows);
+        geo.n_mt = (n_rows_act + 2 * BLOCK_M - 1) / (2 * BLOCK_M);
+    }
+    const int n_tiles = geo.n_mt * geo.n_vt;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (each CTA)
@@ -286,7 +293,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty0 + (uint32_t)acc * 8);
             const int row = m_tile * 256 + (int)rank * BLOCK_M + row_in_tile;
-            if (row < n_rows) {
+            if (row < n_rows_act) {
                 const size_t o = (size_t)v_tile * n_rows + row;
                 pm[o] = run_m;
                 ps[o] = run_s;
@@ -308,7 +315,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 }  // namespace
 
 int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
-                          int32_t* status_dev, cudaStream_t st) {
+                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(confidence_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES) !=
@@ -338,7 +345,7 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc2_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
-                                       part.s, part.a, status_dev);
+                                       part.s, part.a, status_dev, n_rows_dev);
     count_launch();
     if (e != cudaSuccess) return PSD_ERR_CUDA;
     return g.n_vt;

@@ -248,6 +248,7 @@ struct StepTailArgs {
     const float* ps;
     const int32_t* pa;
     int n_split, n_rows, M;
+    const int32_t* pos;   // NULL, or the column of each row's partials when rows were compacted
     psd_policy_t p;
     int32_t* tokV;
     float* confV;
@@ -279,7 +280,7 @@ __global__ void step_tail_kernel(const StepTailArgs a) {
         const int r0 = c < n_chunks ? row_begin + c * kCombineRows : row_end;
         if (grp < groups)
             combine_rows32(a.pm, a.ps, a.pa, a.n_split, a.n_rows, r0, row_end, g, sh[grp], a.tokV, a.confV,
-                           nullptr);
+                           nullptr, a.pos);
     }
     __syncthreads();
 
@@ -332,8 +333,10 @@ int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma,
 int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_policy_t p,
                      int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
                      int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
-                     int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st) {
+                     int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st,
+                     const int32_t* pos) {
     StepTailArgs a;
+    a.pos = pos;
     a.pm = part.m; a.ps = part.s; a.pa = part.a;
     a.n_split = n_split; a.n_rows = n_rows; a.M = M; a.p = p;
     a.tokV = tokV; a.confV = confV;

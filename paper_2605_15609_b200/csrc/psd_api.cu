@@ -11,6 +11,7 @@ std::atomic<int> g_conf_impl{0};
 std::atomic<int> g_pdl{1};
 std::atomic<int> g_band_bytes{36 << 20};
 std::atomic<int> g_tile_order{0};
+std::atomic<int> g_compact{0};
 thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -36,11 +37,11 @@ long long band_bytes() { return g_band_bytes.load(std::memory_order_relaxed); }
 int tile_order() { return g_tile_order.load(std::memory_order_relaxed); }
 
 int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
-                         int32_t* status_dev, cudaStream_t st) {
+                         int32_t* status_dev, cudaStream_t st, const int32_t* n_rows_dev) {
     const int impl = g_conf_impl.load(std::memory_order_relaxed);
     const bool pairs = impl == 3;   // the single-CTA kernel measured faster at every size (see confidence_tc2.cu)
-    return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, st)
-                 : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, st);
+    return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st)
+                 : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st);
 }
 }  // namespace psd
 
@@ -68,6 +69,11 @@ size_t psd_workspace_bytes(int32_t n_rows, int32_t H, int32_t V) {
     return round_up((size_t)max_splits(V) * (size_t)n_rows * 12, 256);
 }
 
+size_t psd_compact_workspace_bytes(int32_t n_rows, int32_t H, int32_t V) {
+    if (!conf_shape_ok(n_rows, H, V)) return 0;
+    return partial_bytes(n_rows, V) + compact_extra_bytes(n_rows, H);
+}
+
 int psd_set_confidence_impl(int impl) {
     if (impl < 0 || impl > 3) return PSD_ERR_SHAPE;
     return g_conf_impl.exchange(impl);
@@ -82,6 +88,10 @@ int psd_set_tuning(int knob, int value) {
         case PSD_TUNE_TILE_ORDER:
             if (value < 0 || value > 2) return PSD_ERR_SHAPE;
             g_tile_order.store(value);
+            return PSD_OK;
+        case PSD_TUNE_COMPACT_ROWS:
+            if (value < 0 || value > 2) return PSD_ERR_SHAPE;
+            g_compact.store(value);
             return PSD_OK;
         case PSD_TUNE_PDL:
             if (value != 0 && value != 1) return PSD_ERR_SHAPE;
@@ -105,14 +115,21 @@ int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t
                    int32_t* out_token, float* out_conf, float* out_lse,
                    void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
     if (!hidden_bf16 || !w_lm_bf16 || !out_token || !out_conf || !workspace) return PSD_ERR_NULL;
-    if (row_ids) return PSD_ERR_UNSUPPORTED;
     if (!conf_shape_ok(n_rows, H, V)) return PSD_ERR_SHAPE;
     if (!aligned(hidden_bf16, 16) || !aligned(w_lm_bf16, 16) || !aligned(workspace, 256) ||
-        !aligned(out_token, 4) || !aligned(out_conf, 4) || !aligned(out_lse, 4) || !aligned(status_dev, 4))
+        !aligned(out_token, 4) || !aligned(out_conf, 4) || !aligned(out_lse, 4) || !aligned(status_dev, 4) ||
+        !aligned(row_ids, 4))
         return PSD_ERR_ALIGN;
-    if (workspace_bytes < psd_workspace_bytes(n_rows, H, V)) return PSD_ERR_WORKSPACE;
+    if (workspace_bytes < (row_ids ? psd_compact_workspace_bytes(n_rows, H, V) : psd_workspace_bytes(n_rows, H, V)))
+        return PSD_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     Partials part = carve_partials(workspace, n_rows, V);
+    if (row_ids) {
+        // the listed rows are copied into a dense buffer first; everything after is the dense path
+        CompactSpace cs = carve_compact(workspace, n_rows, H, V);
+        if (int e = launch_gather_rows(hidden_bf16, row_ids, nullptr, n_rows, n_rows, H, cs.hidden, st)) return e;
+        hidden_bf16 = cs.hidden;
+    }
     const bool timed = t_ev_start && t_ev_stop;
     if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
     int n_split = g_conf_impl.load() == 1
@@ -183,16 +200,33 @@ int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V
     if (!aligned(io->hidden_bf16, 16) || !aligned(io->w_lm_bf16, 16) || !aligned(workspace, 256) ||
         !aligned(status_dev, 4))
         return PSD_ERR_ALIGN;
-    if (workspace_bytes < psd_workspace_bytes(n_rows, H, V)) return PSD_ERR_WORKSPACE;
+    const int compact_mode = g_compact.load(std::memory_order_relaxed);
+    const bool compact = compact_mode == 2 || (compact_mode == 1 && n_rows > 128);
+    if (workspace_bytes < (compact ? psd_compact_workspace_bytes(n_rows, H, V) : psd_workspace_bytes(n_rows, H, V)))
+        return PSD_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     Partials part = carve_partials(workspace, n_rows, V);
+    const void* hidden = io->hidden_bf16;
+    const int32_t* pos = nullptr;
+    const int32_t* n_rows_dev = nullptr;
+    if (compact) {
+        // Only the rows of slots still masked in their draft are scored (Stage 3 needs no others): list
+        // them, copy their hidden states into a dense buffer, and let the fused kernel read the count
+        // from the device, so the step still needs no host synchronisation.
+        CompactSpace cs = carve_compact(workspace, n_rows, H, V);
+        if (int e = launch_list_rows(io->draft_mask, n_rows, cs.row_ids, cs.pos, cs.count, st)) return e;
+        if (int e = launch_gather_rows(hidden, cs.row_ids, cs.count, 0, n_rows, H, cs.hidden, st)) return e;
+        hidden = cs.hidden;
+        pos = cs.pos;
+        n_rows_dev = cs.count;
+    }
     // Two launches: the fused LM-head + confidence kernel, then one kernel per sequence block that
     // merges the split-V partials and runs acceptance, the policy on node k* and the next drafts.
     const bool timed = t_ev_start && t_ev_stop;
     if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
     int n_split = g_conf_impl.load() == 1
-                      ? launch_confidence_simt(io->hidden_bf16, io->w_lm_bf16, n_rows, H, V, part, st)
-                      : launch_confidence_tc(io->hidden_bf16, io->w_lm_bf16, n_rows, H, V, part, status_dev, st);
+                      ? launch_confidence_simt(hidden, io->w_lm_bf16, n_rows, H, V, part, st)
+                      : launch_confidence_tc(hidden, io->w_lm_bf16, n_rows, H, V, part, status_dev, st, n_rows_dev);
     if (timed) {
         cudaError_t ce = cudaEventRecord(t_ev_stop, st);
         t_ev_start = t_ev_stop = nullptr;
@@ -201,7 +235,7 @@ int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V
     if (n_split < 0) return n_split;
     return launch_step_tail(part, n_split, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
                             io->draft_tokens, io->draft_mask, io->tokens, io->mask, io->k_star,
-                            io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st);
+                            io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st, pos);
 }
 
 // Device staging layout of psd_step_host, in order; every piece 256-byte aligned.

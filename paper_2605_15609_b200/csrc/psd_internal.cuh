@@ -41,16 +41,47 @@ int launch_confidence_simt(const void* hidden, const void* w, int n_rows, int H,
 
 // Tensor-core kernels (tcgen05 + TMA).  Each returns the number of splits written, or < 0 (psd_status).
 // confidence_tc.cu: one CTA per tile of 128 rows; confidence_tc2.cu: a pair of CTAs per tile of 256 rows.
+// n_rows_dev: NULL, or a device word holding how many of the n_rows rows actually hold data (the rest
+// of the buffer is ignored; n_rows stays the capacity and the stride of the partial arrays).
 int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V,
-                          Partials part, int32_t* status_dev, cudaStream_t st);
+                          Partials part, int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st);
 int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V,
-                          Partials part, int32_t* status_dev, cudaStream_t st);
+                          Partials part, int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st);
 // psd_api.cu: picks the kernel according to psd_set_confidence_impl.
 int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V,
-                         Partials part, int32_t* status_dev, cudaStream_t st);
+                         Partials part, int32_t* status_dev, cudaStream_t st, const int32_t* n_rows_dev = nullptr);
 
 long long band_bytes();   // psd_api.cu: L2 budget for the operand that a band of the tile order keeps resident
 int tile_order();         // psd_api.cu: 0 = choose, 1 = vocabulary bands, 2 = row bands
+
+// compact.cu: ordered list of the rows whose flag is set (row_ids, inverse map pos, count on the device),
+// and a gather of those rows of a [*, H] bf16 matrix into a dense buffer.
+int launch_list_rows(const int32_t* flags, int n, int32_t* row_ids, int32_t* pos, int32_t* count, cudaStream_t st);
+int launch_gather_rows(const void* src, const int32_t* row_ids, const int32_t* count_dev, int count_host, int max_rows,
+                       int H, void* dst, cudaStream_t st);
+
+// Extra workspace of the compacted path, after the partial triples: dense hidden rows, row list,
+// inverse map, count.
+struct CompactSpace {
+    void* hidden;       // [n_rows, H] bf16
+    int32_t* row_ids;   // [n_rows]
+    int32_t* pos;       // [n_rows]
+    int32_t* count;     // [1]
+};
+inline size_t partial_bytes(int n_rows, int V) { return ((size_t)max_splits(V) * (size_t)n_rows * 12 + 255) / 256 * 256; }
+inline size_t compact_extra_bytes(int n_rows, int H) {
+    return ((size_t)n_rows * H * 2 + 255) / 256 * 256 + ((size_t)n_rows * 8 + 4 + 255) / 256 * 256;
+}
+inline CompactSpace carve_compact(void* workspace, int n_rows, int H, int V) {
+    unsigned char* p = reinterpret_cast<unsigned char*>(workspace) + partial_bytes(n_rows, V);
+    CompactSpace c;
+    c.hidden = p;
+    p += ((size_t)n_rows * H * 2 + 255) / 256 * 256;
+    c.row_ids = reinterpret_cast<int32_t*>(p);
+    c.pos = c.row_ids + n_rows;
+    c.count = c.pos + n_rows;
+    return c;
+}
 
 // combine.cu: merge n_split partial triples per row.
 int launch_combine(Partials part, int n_split, int n_rows,
@@ -73,6 +104,7 @@ int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma,
 int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_policy_t p,
                      int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
                      int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
-                     int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st);
+                     int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st,
+                     const int32_t* pos = nullptr);
 
 }  // namespace psd

@@ -69,7 +69,11 @@ def test_confidence_argument_errors():
     assert _conf(w=None) == psd.PSD_ERR_NULL
     assert _conf(tok=None) == psd.PSD_ERR_NULL
     assert _conf(ws=None) == psd.PSD_ERR_NULL
-    assert _conf(row_ids=FAKE) == psd.PSD_ERR_UNSUPPORTED
+    # a row list needs the larger workspace (room for the dense copy of the listed rows)
+    assert _conf(row_ids=FAKE, ws_bytes=psd.psd_workspace_bytes(128, 256, 1024)) == psd.PSD_ERR_WORKSPACE
+    assert _conf(row_ids=FAKE + 2, ws_bytes=1 << 30) == psd.PSD_ERR_ALIGN
+    assert psd.psd_compact_workspace_bytes(128, 256, 1024) >= psd.psd_workspace_bytes(128, 256, 1024) + 128 * 256 * 2
+    assert psd.psd_compact_workspace_bytes(0, 256, 1024) == 0
     assert _conf(n_rows=0) == psd.PSD_ERR_SHAPE
     assert _conf(H=100) == psd.PSD_ERR_SHAPE
     assert _conf(H=0) == psd.PSD_ERR_SHAPE

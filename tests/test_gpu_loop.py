@@ -40,7 +40,7 @@ class Loop:
         self.max_it = max_iterations or (M + 2)
         hidden = torch.zeros(B * D * M, H, dtype=torch.bfloat16, device="cuda")
         self.buf = psd.StepBuffers.allocate(B, M, D, H, hidden, self.w_dev, "cuda")
-        self.ws = torch.empty(psd.psd_workspace_bytes(B * D * M, H, V), dtype=torch.uint8, device="cuda")
+        self.ws = torch.empty(psd.psd_compact_workspace_bytes(B * D * M, H, V), dtype=torch.uint8, device="cuda")
         self.scratch = torch.empty(psd.psd_decode_scratch_bytes(B, M), dtype=torch.uint8, device="cuda")
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.passes = torch.zeros(B, dtype=torch.int32, device="cuda")
@@ -167,6 +167,19 @@ def test_loop_matches_oracle(name, order):
     if loop.cfg.D > 1:
         assert max(k_stars) > 0                      # some speculation was accepted
         assert stats.iterations < loop.cfg.M         # fewer iterations than slots
+
+
+@pytest.mark.parametrize("name", ["threshold", "long_block"])
+def test_loop_with_row_compaction(name):
+    """The one-pass loop with psd_step scoring only masked rows: same parity bar."""
+    loop = Loop(CASES[name])
+    assert psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, 2) == 0
+    try:
+        stats = loop.run_native(psd.ORDER_ONE_PASS)
+    finally:
+        psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, 0)
+    set_aside, _, k_stars = loop.compare(psd.ORDER_ONE_PASS, stats)
+    assert set_aside <= loop.cfg.B // 2 and max(k_stars) > 0
 
 
 @pytest.mark.parametrize("order", [psd.ORDER_TWO_PASSES, psd.ORDER_ONE_PASS])
