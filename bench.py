@@ -322,7 +322,7 @@ def run_ours(args, cfg):
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside)
     hv_host = bf16(wl.hidden_verify, pin=True)
-    hb = psd.StepBuffers.allocate(B, M, D, H, hv_host, w_dev, "cpu", pin=True)
+    hb = psd.host_step_buffers(B, M, D, hv_host, w_dev)     # one pinned block: single copies each way
     for k, v in first.items():
         getattr(hb, k).copy_(v)
     staging = torch.empty(psd.psd_step_host_bytes(B, M, H, V, D), dtype=torch.uint8, device=device)
@@ -331,8 +331,11 @@ def run_ours(args, cfg):
         psd.psd_step_host(hb, pg, staging, stream)
     secs_e2e = timed_region(lambda i: psd.psd_step_host(hb, pg, staging, stream), n_e2e)
     e2e_value, _ = replicas.aggregate_throughput(float(R) * n_e2e, secs_e2e, info, device)
-    h2d = R * H * 2 + 4 * (B * M + B * D + 2 * R)
-    d2h = 4 * (B * M + B * D + 2 * R) + 4 * (2 * R) + 4 * (2 * B * M) + 4 * (3 * B) + 4 * (2 * B * M + B) + 4
+    # bytes actually moved per step: hidden plus the draft state up (one block, padding included), every
+    # output and the status word down (one block)
+    _, off = psd.psd_step_host_block(B, M, D)
+    h2d = R * H * 2 + off[4]
+    d2h = off[14] + 4
 
     if not info.is_main:
         return 0

@@ -255,6 +255,17 @@ int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V
 size_t psd_step_host_bytes(int32_t B, int32_t M, int32_t H, int32_t V, int32_t D);
 
 /*
+ * Layout of ONE host block that holds every per-step array of psd_step_io_t except hidden_bf16 and
+ * w_lm_bf16.  Returns the block's size in bytes (0 for invalid sizes) and, if offsets != NULL, the 15
+ * byte offsets of sigma, n_fill, draft_tokens, draft_mask, tokV, confV, tokens, mask, k_star,
+ * n_spec_accepted, n_committed, sel, n_sel, sel_pos and of a status word, in this order.  When the
+ * io passed to psd_step_host points into such a block (pinned memory recommended), the draft state
+ * is copied up in one transfer and all outputs come back in one; any other arrangement of host
+ * arrays works too, with one transfer per array.
+ */
+size_t psd_step_host_block(int32_t B, int32_t M, int32_t D, size_t* offsets);
+
+/*
  * psd_step_host — psd_step for callers whose per-step data lives in host memory.
  * Copies hidden and the draft state host->device into `staging`, runs psd_step, copies every
  * output of io back device->host, and waits for the stream.  io holds HOST pointers

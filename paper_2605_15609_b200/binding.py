@@ -91,6 +91,8 @@ def _load() -> ctypes.CDLL:
     lib.psd_step.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
     lib.psd_step_host_bytes.restype = _sz
     lib.psd_step_host_bytes.argtypes = [_i32, _i32, _i32, _i32, _i32]
+    lib.psd_step_host_block.restype = _sz
+    lib.psd_step_host_block.argtypes = [_i32, _i32, _i32, ctypes.POINTER(_sz)]
     lib.psd_step_host.restype = ctypes.c_int
     lib.psd_step_host.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _vp, _sz, _vp, _vp]
     lib.psd_dag_init.restype = ctypes.c_int
@@ -277,6 +279,33 @@ class StepBuffers:
                            confV=torch.zeros(B, D, M, dtype=torch.float32, **kw), tokens=i32(B, M), mask=i32(B, M),
                            k_star=i32(B), n_spec_accepted=i32(B), n_committed=i32(B), sel=i32(B, M), n_sel=i32(B),
                            sel_pos=i32(B, M))
+
+
+def psd_step_host_block(B, M, D):
+    """(bytes, offsets[15]) of the one-block host layout that psd_step_host moves with single copies."""
+    off = (_sz * 15)()
+    n = int(LIB.psd_step_host_block(B, M, D, off))
+    return n, [int(x) for x in off]
+
+
+def host_step_buffers(B, M, D, hidden, w_lm) -> StepBuffers:
+    """StepBuffers whose arrays are views of ONE pinned host block laid out as psd_step_host_block says
+    (``hidden``: a host tensor, ``w_lm``: a device tensor).  The block is kept alive by the views."""
+    n, off = psd_step_host_block(B, M, D)
+    block = torch.zeros(n, dtype=torch.uint8).pin_memory()
+
+    def view(o, shape, dtype=torch.int32):
+        count = 1
+        for d in shape:
+            count *= d
+        return block[o:o + 4 * count].view(dtype).view(*shape)
+
+    return StepBuffers(hidden=hidden, w_lm=w_lm, sigma=view(off[0], (B, M)), n_fill=view(off[1], (B, D)),
+                       draft_tokens=view(off[2], (B, D, M)), draft_mask=view(off[3], (B, D, M)),
+                       tokV=view(off[4], (B, D, M)), confV=view(off[5], (B, D, M), torch.float32),
+                       tokens=view(off[6], (B, M)), mask=view(off[7], (B, M)), k_star=view(off[8], (B,)),
+                       n_spec_accepted=view(off[9], (B,)), n_committed=view(off[10], (B,)), sel=view(off[11], (B, M)),
+                       n_sel=view(off[12], (B,)), sel_pos=view(off[13], (B, M)))
 
 
 def psd_step(buf: StepBuffers, p: PsdPolicy, workspace, status=None, stream=None):

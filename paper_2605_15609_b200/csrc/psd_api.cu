@@ -271,6 +271,17 @@ Staging staging_layout(int B, int M, int H, int V, int D) {
 }
 }  // namespace
 
+size_t psd_step_host_block(int32_t B, int32_t M, int32_t D, size_t* offsets) {
+    if (check_block_shape(B, M) || D < 1 || D > PSD_MAX_DEPTH || (long long)B * D * M > 2147483647ll) return 0;
+    // H and V only size pieces outside [sigma, status]: any valid pair gives the same offsets in between
+    const Staging s = staging_layout(B, M, 64, 1, D);
+    const size_t at[15] = {s.sigma, s.n_fill, s.draft_tokens, s.draft_mask, s.tokV, s.confV, s.tokens, s.mask,
+                           s.k_star, s.n_spec, s.n_comm, s.sel, s.n_sel, s.sel_pos, s.status};
+    if (offsets)
+        for (int i = 0; i < 15; ++i) offsets[i] = at[i] - s.sigma;
+    return s.status + 256 - s.sigma;
+}
+
 size_t psd_step_host_bytes(int32_t B, int32_t M, int32_t H, int32_t V, int32_t D) {
     if (check_block_shape(B, M) || D < 1 || D > PSD_MAX_DEPTH || (long long)B * D * M > 2147483647ll) return 0;
     if (!conf_shape_ok(B * D * M, H, V)) return 0;
@@ -293,6 +304,15 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     const size_t R = (size_t)B * D * M, BM = (size_t)B * M;
     bool ok = true;
+    // One block: when the caller's arrays sit in host memory exactly as psd_step_host_block lays them
+    // out, the draft state goes up in one copy and every output comes back in one.
+    const unsigned char* hb = reinterpret_cast<const unsigned char*>(io->sigma);
+    auto at = [&](const void* ptr, size_t off) { return reinterpret_cast<const unsigned char*>(ptr) == hb + (off - s.sigma); };
+    const bool one_block = at(io->n_fill, s.n_fill) && at(io->draft_tokens, s.draft_tokens) &&
+                           at(io->draft_mask, s.draft_mask) && at(io->tokV, s.tokV) && at(io->confV, s.confV) &&
+                           at(io->tokens, s.tokens) && at(io->mask, s.mask) && at(io->k_star, s.k_star) &&
+                           at(io->n_spec_accepted, s.n_spec) && at(io->n_committed, s.n_comm) && at(io->sel, s.sel) &&
+                           at(io->n_sel, s.n_sel) && at(io->sel_pos, s.sel_pos);
     auto h2d = [&](size_t off, const void* src, size_t bytes) {
         ok = ok && cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
     };
@@ -300,10 +320,14 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
         ok = ok && cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     };
     h2d(s.hidden, io->hidden_bf16, R * H * 2);
-    h2d(s.sigma, io->sigma, BM * 4);
-    h2d(s.n_fill, io->n_fill, (size_t)B * D * 4);
-    h2d(s.draft_tokens, io->draft_tokens, R * 4);
-    h2d(s.draft_mask, io->draft_mask, R * 4);
+    if (one_block) {
+        h2d(s.sigma, io->sigma, s.tokV - s.sigma);
+    } else {
+        h2d(s.sigma, io->sigma, BM * 4);
+        h2d(s.n_fill, io->n_fill, (size_t)B * D * 4);
+        h2d(s.draft_tokens, io->draft_tokens, R * 4);
+        h2d(s.draft_mask, io->draft_mask, R * 4);
+    }
     ok = ok && cudaMemsetAsync(d + s.status, 0, 4, st) == cudaSuccess;
     if (!ok) return PSD_ERR_CUDA;
 
@@ -328,6 +352,14 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
                      reinterpret_cast<int32_t*>(d + s.status), cuda_stream);
     if (e) return e;
 
+    if (one_block) {
+        // [sigma .. status]: the status word lands in the caller's block, at the offset the layout gives it
+        d2h(io->sigma, s.sigma, s.status + 4 - s.sigma);
+        ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+        if (!ok) return PSD_ERR_CUDA;
+        if (status_host) *status_host = *reinterpret_cast<const int32_t*>(hb + (s.status - s.sigma));
+        return PSD_OK;
+    }
     d2h(io->sigma, s.sigma, BM * 4);
     d2h(io->n_fill, s.n_fill, (size_t)B * D * 4);
     d2h(io->draft_tokens, s.draft_tokens, R * 4);

@@ -130,8 +130,9 @@ def test_psd_step_equals_the_four_calls_and_is_deterministic():
         assert np.array_equal(v.cpu().numpy(), runs[0][k]), k
 
 
+@pytest.mark.parametrize("one_block", [False, True])
 @pytest.mark.parametrize("name", ["tiny", "single_request"])
-def test_psd_step_host_matches_device_step(name):
+def test_psd_step_host_matches_device_step(name, one_block):
     cfg, wl, w_dev = _workload(name)
     po, pg = policies(cfg)
     B, M, D = cfg.B, cfg.M, cfg.D
@@ -140,7 +141,12 @@ def test_psd_step_host_matches_device_step(name):
     want = gpu_step(step_buffers_from(chain, cfg, hv_dev, w_dev), cfg, pg)
 
     hv_host = hv_dev.cpu().pin_memory()
-    hb = psd.StepBuffers.allocate(B, M, D, cfg.H, hv_host, w_dev, "cpu", pin=True)
+    if one_block:   # every array a view of one pinned block: single copies in each direction
+        hb = psd.host_step_buffers(B, M, D, hv_host, w_dev)
+        n, off = psd.psd_step_host_block(B, M, D)
+        assert hb.n_fill.data_ptr() - hb.sigma.data_ptr() == off[1] and off[0] == 0 and n >= off[14] + 4
+    else:
+        hb = psd.StepBuffers.allocate(B, M, D, cfg.H, hv_host, w_dev, "cpu", pin=True)
     hb.sigma.copy_(chain.sigma)
     hb.n_fill.copy_(chain.n_fill)
     hb.draft_tokens.copy_(chain.draft_tokens)
