@@ -304,8 +304,9 @@ def verify_accept(tokV, confV, sigma, n_fill, draft_tokens, draft_mask, p: Polic
     return tokens, mask, k_star, n_spec, n_comm, accepted
 
 
-def decode_block(model, M: int, p: Policy, max_steps: int | None = None):
-    """Algorithm 1 for one block.
+def decode_block(model, M: int, p: Policy, max_steps: int | None = None, node_ranks=None, edges=None):
+    """Algorithm 1 for one block.  With node_ranks (and optionally edges) the drafts form that graph
+    instead of the chain of p.depth nodes.
 
     ``model(tokens[K, M], mask[K, M]) -> (tok[K, M], conf[K, M])`` stands for p_theta.
     Returns the final tokens, the number of model calls, and a per-iteration log of
@@ -322,26 +323,34 @@ def decode_block(model, M: int, p: Policy, max_steps: int | None = None):
         tok, conf = model(tokens, mask)
         calls += 1
         tokens, mask, _, n_sel, _ = select_unmask(conf, tok, tokens, mask, p)
-        if not mask.any() or p.depth == 1:
+        if not mask.any() or (p.depth == 1 if node_ranks is None else len(node_ranks) == 1):
             # the block is resolved (Algorithm 1's early break), or there is nothing to speculate:
             # a chain of the root alone is plain spatial decoding, one model call per iteration
             log.append((int(n_sel[0]), 0, 0, 0))
             continue
-        sigma, n_fill, dt, dm = build_drafts(conf, tok, tokens, mask, p)
+        if node_ranks is None:
+            sigma, n_fill, dt, dm = build_drafts(conf, tok, tokens, mask, p)
+        else:
+            sigma, n_fill, dt, dm = build_drafts_dag(conf, tok, tokens, mask, p, node_ranks)
         tv, cv = model(dt[0], dm[0])
         calls += 1
-        tokens, mask, ks, ns, nc, _ = verify_accept(np.asarray(tv)[None], np.asarray(cv)[None],
-                                                    sigma, n_fill, dt, dm, p)
+        if node_ranks is None:
+            tokens, mask, ks, ns, nc, _ = verify_accept(np.asarray(tv)[None], np.asarray(cv)[None],
+                                                        sigma, n_fill, dt, dm, p)
+        else:
+            tokens, mask, ks, ns, nc, _ = verify_accept_dag(np.asarray(tv)[None], np.asarray(cv)[None],
+                                                            sigma, dt, dm, p, node_ranks, edges)
         log.append((int(n_sel[0]), int(ks[0]), int(ns[0]), int(nc[0])))
     return tokens[0], calls, log
 
 
-def decode_block_one_pass(model, M: int, p: Policy, max_steps: int | None = None):
+def decode_block_one_pass(model, M: int, p: Policy, max_steps: int | None = None, node_ranks=None, edges=None):
     """Algorithm 1 rearranged so that every iteration costs ONE model call.
 
     The batched pass on the D drafts also scores the root (the current state) and every accepted
     node, so its predictions for node k* are exactly what Stage 1 of the next iteration would
-    compute on the state that acceptance leaves behind.  An iteration is therefore:
+    compute on the state that acceptance leaves behind (node_ranks / edges: drafts form that graph
+    instead of the chain).  An iteration is therefore:
     model(drafts) -> Stage 3 (acceptance and its extra commit) -> Stage 1 (policy on node k*'s
     predictions, Eq. (1)) -> Stage 2 (next drafts from the same predictions).  The first iteration
     verifies D copies of the initial state with nothing speculated.  This is an arrangement of the
@@ -351,7 +360,7 @@ def decode_block_one_pass(model, M: int, p: Policy, max_steps: int | None = None
     (|T|, k*, n_spec_accepted, n_committed).
     """
     p.check()
-    D = p.depth
+    D = p.depth if node_ranks is None else len(node_ranks)
     tokens = np.full((1, M), p.mask_id, dtype=np.int32)
     mask = np.ones((1, M), dtype=np.int32)
     sigma = np.full((1, M), -1, dtype=np.int32)
@@ -366,10 +375,16 @@ def decode_block_one_pass(model, M: int, p: Policy, max_steps: int | None = None
         tv, cv = model(dt[0], dm[0])
         calls += 1
         tv, cv = np.asarray(tv)[None], np.asarray(cv, dtype=np.float64)[None]
-        tokens, mask, ks, ns, nc, _ = verify_accept(tv, cv, sigma, n_fill, dt, dm, p)
+        if node_ranks is None:
+            tokens, mask, ks, ns, nc, _ = verify_accept(tv, cv, sigma, n_fill, dt, dm, p)
+        else:
+            tokens, mask, ks, ns, nc, _ = verify_accept_dag(tv, cv, sigma, dt, dm, p, node_ranks, edges)
         ck, tk = cv[:, int(ks[0])], tv[:, int(ks[0])]
         tokens, mask, _, n_sel, _ = select_unmask(ck, tk, tokens, mask, p)
-        sigma, n_fill, dt, dm = build_drafts(ck, tk, tokens, mask, p)
+        if node_ranks is None:
+            sigma, n_fill, dt, dm = build_drafts(ck, tk, tokens, mask, p)
+        else:
+            sigma, n_fill, dt, dm = build_drafts_dag(ck, tk, tokens, mask, p, node_ranks)
         log.append((int(n_sel[0]), int(ks[0]), int(ns[0]), int(nc[0])))
     return tokens[0], calls, log
 

@@ -12,7 +12,7 @@ LIB = os.path.join(PKG, "libpsd_b200.so")
 SOURCES = ["psd_api.cu", "confidence_tc.cu", "confidence_tc2.cu", "confidence_simt.cu", "combine.cu", "policy.cu",
            "confidence_static.cu", "decode_loop.cu", "dag.cu", "compact.cu"]
 EXTRA_SOURCES: list[str] = []
-NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+NVCC_FLAGS = [*os.environ.get("PSD_NVCC_EXTRA", "").split(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 

@@ -14,7 +14,10 @@ constexpr int BLOCK_M = 128;       // rows per tile (TMEM lanes)
 constexpr int BLOCK_N = 256;       // widest vocabulary tile (TMEM columns per accumulator)
 constexpr int BLOCK_K = 64;        // bf16 elements per K-slice = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
+#ifndef PSD_STAGES
+#define PSD_STAGES 4
+#endif
+constexpr int STAGES = PSD_STAGES;   // depth of the shared-memory ring (48 KB per stage)
 constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;   // 16 KB
 constexpr int B_BYTES = BLOCK_N * BLOCK_K * 2;   // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;

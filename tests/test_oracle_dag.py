@@ -142,3 +142,37 @@ def test_structure_and_truncation():
     with pytest.raises(ValueError):
         oracle.verify_accept_dag(np.zeros((B, 5, M), int), np.zeros((B, 5, M)), sigma, dt, dm, p, node_ranks,
                                  edges=[(1, 3)])
+
+
+class _Stable:
+    """A model whose predictions never change: target tokens, confidence falling with the slot index."""
+
+    def __init__(self, M):
+        self.target = np.arange(100, 100 + M, dtype=np.int32)
+        self.calls = []
+
+    def __call__(self, tokens, mask):
+        mask = np.atleast_2d(mask)
+        self.calls.append(mask.shape[0])
+        conf = np.tile(0.8 - 0.03 * np.arange(mask.shape[1]), (mask.shape[0], 1))
+        return np.tile(self.target, (mask.shape[0], 1)), conf
+
+
+@pytest.mark.parametrize("loop", [oracle.decode_block, oracle.decode_block_one_pass])
+def test_loops_with_a_path_graph_equal_the_chain_loops(loop):
+    M, D = 14, 4
+    p = Policy(tau=1.0, k_min=1, k_max=1, depth=D, accept_mode=1, mask_id=MASK)
+    chain = loop(_Stable(M), M, p)
+    graph = loop(_Stable(M), M, p, node_ranks=oracle.chain_as_dag(D, 1), edges=[(d - 1, d) for d in range(1, D)])
+    assert (chain[0] == graph[0]).all() and chain[1] == graph[1] and chain[2] == graph[2]
+
+
+def test_loop_with_a_wider_graph_commits_every_slot_once():
+    M = 20
+    ranks = [set(), {0}, {1}, {0, 1}, {0, 1, 2}, {0, 2}]
+    p = Policy(tau=0.5, k_min=1, k_max=3, depth=1, accept_mode=1, mask_id=MASK)
+    for loop in (oracle.decode_block, oracle.decode_block_one_pass):
+        m = _Stable(M)
+        tokens, calls, log = loop(m, M, p, node_ranks=ranks)
+        assert (tokens == m.target).all() and sum(n + nc for n, _, _, nc in log) == M
+        assert max(ks for _, ks, _, _ in log) > 0 and set(m.calls) <= {1, len(ranks)}
