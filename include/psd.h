@@ -329,6 +329,15 @@ int psd_verify_accept_dag(const int32_t* tokV, const float* confV, const int32_t
                           int32_t* n_spec_accepted, int32_t* n_committed, int32_t* accepted, void* cuda_stream);
 
 /*
+ * psd_step_dag — psd_step with the drafts of a graph: D = g->n_nodes in every shape of io; acceptance is
+ * psd_verify_accept_dag, the next drafts psd_build_drafts_dag (p.depth and p.stride are not used).
+ * Runs as separate launches (fused kernel, merge, acceptance, policy, drafts) on the stream.
+ */
+int psd_step_dag(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+                 const psd_dag_t* g, void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                 void* cuda_stream);
+
+/*
  * ---- The whole decoding loop of Algorithm 1 over a batch of blocks ----------------------------------
  *
  * The transformer body is the caller's: a function that, given token states on the device, writes
@@ -366,6 +375,8 @@ size_t psd_decode_scratch_bytes(int32_t B, int32_t M);
  * psd_step_io_t; after the call they hold the last iteration's values.  D = p.depth; with D = 1
  * nothing is speculated and every iteration is one pass (plain parallel decoding).
  *
+ *   g               NULL: the drafts are the chain of p.depth nodes; else a draft graph (HOST pointer),
+ *                   and D = g->n_nodes in every shape above (p.depth, p.stride are then not used)
  *   order           PSD_ORDER_TWO_PASSES or PSD_ORDER_ONE_PASS
  *   scratch         device, 256-byte aligned, >= psd_decode_scratch_bytes(B, M)
  *   workspace       as for psd_confidence with n_rows = B*D*M
@@ -381,7 +392,7 @@ size_t psd_decode_scratch_bytes(int32_t B, int32_t M);
  * 4-byte copy and a stream synchronisation) to decide whether to go on.  It allocates nothing.
  */
 int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int32_t B, int32_t M, int32_t H,
-                      int32_t V, psd_policy_t p, int32_t order, int32_t max_iterations,
+                      int32_t V, psd_policy_t p, const psd_dag_t* g, int32_t order, int32_t max_iterations,
                       void* scratch, size_t scratch_bytes, void* workspace, size_t workspace_bytes,
                       int32_t* status_dev, int32_t* passes, int32_t* done_iteration, int32_t* trace,
                       psd_decode_stats_t* stats, void* cuda_stream);

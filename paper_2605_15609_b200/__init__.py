@@ -12,7 +12,7 @@ from .binding import (ACCEPT_AGREE_AND_CONF, ACCEPT_AGREE_AND_POLICY, ACCEPT_AGR
                       psd_launch_count, psd_select_unmask, psd_set_confidence_impl, psd_set_kernel_events, psd_set_tuning, PSD_TUNE_BAND_BYTES, PSD_TUNE_PDL, PSD_TUNE_TILE_ORDER, PSD_TUNE_COMPACT_ROWS, psd_compact_workspace_bytes, psd_step, psd_step_host,
                       psd_step_host_bytes, psd_step_host_block, host_step_buffers, psd_verify_accept, psd_workspace_bytes, status_string, psd_decode_blocks, psd_decode_scratch_bytes,
                       table_body_address, table_body_user, psd_table_body, PsdDag, psd_dag_init,
-                      psd_build_drafts_dag, psd_verify_accept_dag, PsdDecodeStats, PsdTableBody, ORDER_TWO_PASSES,
+                      psd_build_drafts_dag, psd_verify_accept_dag, psd_step_dag, PsdDecodeStats, PsdTableBody, ORDER_TWO_PASSES,
                       ORDER_ONE_PASS)
 
 __all__ = [n for n in dir() if not n.startswith("_")]

@@ -106,7 +106,11 @@ def _load() -> ctypes.CDLL:
     lib.psd_decode_scratch_bytes.restype = _sz
     lib.psd_decode_scratch_bytes.argtypes = [_i32, _i32]
     lib.psd_decode_blocks.restype = ctypes.c_int
-    lib.psd_decode_blocks.argtypes = [_vp, _vp, ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, _i32, _i32,
+    lib.psd_step_dag.restype = ctypes.c_int
+    lib.psd_step_dag.argtypes = [ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol, ctypes.POINTER(PsdDag), _vp,
+                                 _sz, _vp, _vp]
+    lib.psd_decode_blocks.argtypes = [_vp, _vp, ctypes.POINTER(PsdStepIO), _i32, _i32, _i32, _i32, pol,
+                                      ctypes.POINTER(PsdDag), _i32, _i32,
                                       _vp, _sz, _vp, _sz, _vp, _vp, _vp, _vp, ctypes.POINTER(PsdDecodeStats), _vp]
     lib.psd_table_body.restype = ctypes.c_int
     lib.psd_table_body.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp]
@@ -338,8 +342,16 @@ def psd_decode_scratch_bytes(B: int, M: int) -> int:
     return int(LIB.psd_decode_scratch_bytes(B, M))
 
 
+def psd_step_dag(buf: StepBuffers, p: PsdPolicy, g: PsdDag, workspace, status=None, stream=None):
+    B, M = buf.tokens.shape
+    io = buf.io()
+    _check(LIB.psd_step_dag(ctypes.byref(io), B, M, buf.hidden.shape[1], buf.w_lm.shape[0], p, ctypes.byref(g),
+                            _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status),
+                            _stream(stream)), "psd_step_dag")
+
+
 def psd_decode_blocks(body, user, buf: StepBuffers, p: PsdPolicy, order: int, max_iterations: int, scratch,
-                      workspace, status=None, passes=None, done_iteration=None, trace=None, stream=None):
+                      workspace, status=None, passes=None, done_iteration=None, trace=None, stream=None, dag=None):
     """Algorithm 1 over the blocks of ``buf`` (device tensors; ``buf.hidden`` is scratch the body fills).
 
     ``body`` is either the address of a native ``psd_body_fn`` (an int, e.g. ``table_body_address()``)
@@ -356,7 +368,8 @@ def psd_decode_blocks(body, user, buf: StepBuffers, p: PsdPolicy, order: int, ma
         cb, body_ptr = None, _vp(int(body))
     io = buf.io()
     stats = PsdDecodeStats()
-    code = LIB.psd_decode_blocks(body_ptr, user, ctypes.byref(io), B, M, H, V, p, int(order), int(max_iterations),
+    code = LIB.psd_decode_blocks(body_ptr, user, ctypes.byref(io), B, M, H, V, p,
+                                 ctypes.byref(dag) if dag is not None else None, int(order), int(max_iterations),
                                  _ptr(scratch), scratch.numel() * scratch.element_size(), _ptr(workspace),
                                  workspace.numel() * workspace.element_size(), _ptr(status), _ptr(passes),
                                  _ptr(done_iteration), _ptr(trace), ctypes.byref(stats), _stream(stream))

@@ -115,7 +115,7 @@ size_t psd_decode_scratch_bytes(int32_t B, int32_t M) {
 }
 
 int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int32_t B, int32_t M, int32_t H,
-                      int32_t V, psd_policy_t p, int32_t order, int32_t max_iterations,
+                      int32_t V, psd_policy_t p, const psd_dag_t* g, int32_t order, int32_t max_iterations,
                       void* scratch, size_t scratch_bytes, void* workspace, size_t workspace_bytes,
                       int32_t* status_dev, int32_t* passes, int32_t* done_iteration, int32_t* trace,
                       psd_decode_stats_t* stats, void* cuda_stream) {
@@ -130,6 +130,10 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
     if (need == 0) return PSD_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(scratch) & 255) return PSD_ERR_ALIGN;
     if (scratch_bytes < need) return PSD_ERR_WORKSPACE;
+    if (g) {
+        if (g->n_nodes < 1 || g->n_nodes > PSD_MAX_DAG_NODES) return PSD_ERR_SHAPE;
+        p.depth = g->n_nodes;     // the drafts are the nodes of the graph
+    }
     const int D = p.depth;
     if (D < 1 || D > PSD_MAX_DEPTH || (long long)B * D * M > 2147483647ll) return PSD_ERR_POLICY;
     if (workspace_bytes < psd_workspace_bytes(B * D * M, H, V) || psd_workspace_bytes(B * D * M, H, V) == 0)
@@ -183,7 +187,9 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
             // one forward pass per iteration: the verification pass of the drafts doubles as the model
             // call of the next iteration (psd_step)
             if ((e = body(user, io->draft_tokens, io->draft_mask, B * D, M, hidden, cuda_stream))) return e;
-            if ((e = psd_step(io, B, M, H, V, p, workspace, workspace_bytes, status_dev, cuda_stream))) return e;
+            e = g ? psd_step_dag(io, B, M, H, V, p, g, workspace, workspace_bytes, status_dev, cuda_stream)
+                  : psd_step(io, B, M, H, V, p, workspace, workspace_bytes, status_dev, cuda_stream);
+            if (e) return e;
             stats->forward_passes += 1;
             record(it, 1);
             if ((e = progress(1, it, &masked))) return e;
@@ -204,17 +210,22 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
                 record(it, 0);
             } else {
                 // Stage 2: drafts from the cached stage-1 predictions.  Stage 3: one batched pass, acceptance.
-                if ((e = psd_build_drafts(conf1, tok1, nullptr, 1, io->tokens, io->mask, B, M, p, io->sigma,
-                                          io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream)))
-                    return e;
+                e = g ? psd_build_drafts_dag(conf1, tok1, nullptr, 1, io->tokens, io->mask, B, M, p, g, io->sigma,
+                                             io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream)
+                      : psd_build_drafts(conf1, tok1, nullptr, 1, io->tokens, io->mask, B, M, p, io->sigma,
+                                         io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream);
+                if (e) return e;
                 if ((e = body(user, io->draft_tokens, io->draft_mask, B * D, M, hidden, cuda_stream))) return e;
                 if ((e = psd_confidence(hidden, io->w_lm_bf16, nullptr, B * D * M, H, V, io->tokV, io->confV, nullptr,
                                         workspace, workspace_bytes, status_dev, cuda_stream)))
                     return e;
-                if ((e = psd_verify_accept(io->tokV, io->confV, io->sigma, io->n_fill, io->draft_tokens,
-                                           io->draft_mask, B, M, p, io->tokens, io->mask, io->k_star,
-                                           io->n_spec_accepted, io->n_committed, nullptr, cuda_stream)))
-                    return e;
+                e = g ? psd_verify_accept_dag(io->tokV, io->confV, io->sigma, io->draft_tokens, io->draft_mask, B, M,
+                                              p, g, io->tokens, io->mask, io->k_star, io->n_spec_accepted,
+                                              io->n_committed, nullptr, cuda_stream)
+                      : psd_verify_accept(io->tokV, io->confV, io->sigma, io->n_fill, io->draft_tokens,
+                                          io->draft_mask, B, M, p, io->tokens, io->mask, io->k_star,
+                                          io->n_spec_accepted, io->n_committed, nullptr, cuda_stream);
+                if (e) return e;
                 stats->forward_passes += 1;
                 record(it, 1);
                 if ((e = progress(1, it, &masked))) return e;

@@ -187,10 +187,16 @@ static int check_step_io(const psd_step_io_t* io) {
     return PSD_OK;
 }
 
-int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
-             void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+// One step for the chain of p.depth nodes (g == NULL) or for the draft graph g.
+static int step_impl(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+                     const psd_dag_t* g, void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                     void* cuda_stream) {
     if (int e = check_step_io(io)) return e;
     if (check_block_shape(B, M)) return PSD_ERR_SHAPE;
+    if (g) {
+        if (g->n_nodes < 1 || g->n_nodes > PSD_MAX_DAG_NODES) return PSD_ERR_SHAPE;
+        p.depth = g->n_nodes;
+    }
     if (int e = check_policy(p)) return e;
     const int D = p.depth;
     if ((long long)B * D * M > 2147483647ll) return PSD_ERR_SHAPE;
@@ -233,9 +239,34 @@ int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V
         if (ce != cudaSuccess) return PSD_ERR_CUDA;
     }
     if (n_split < 0) return n_split;
-    return launch_step_tail(part, n_split, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
-                            io->draft_tokens, io->draft_mask, io->tokens, io->mask, io->k_star,
-                            io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st, pos);
+    if (!g)
+        return launch_step_tail(part, n_split, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
+                                io->draft_tokens, io->draft_mask, io->tokens, io->mask, io->k_star,
+                                io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st, pos);
+    // draft graph: the same stages as separate launches (merge, acceptance over the graph, policy on
+    // node k*, next drafts of the graph)
+    if (int e = launch_combine(part, n_split, n_rows, io->tokV, io->confV, nullptr, st, pos)) return e;
+    if (int e = psd_verify_accept_dag(io->tokV, io->confV, io->sigma, io->draft_tokens, io->draft_mask, B, M, p, g,
+                                      io->tokens, io->mask, io->k_star, io->n_spec_accepted, io->n_committed,
+                                      nullptr, cuda_stream))
+        return e;
+    if (int e = launch_select(io->confV, io->tokV, io->k_star, D, io->tokens, io->mask, B, M, p, io->sel, io->n_sel,
+                              io->sel_pos, st))
+        return e;
+    return psd_build_drafts_dag(io->confV, io->tokV, io->k_star, D, io->tokens, io->mask, B, M, p, g, io->sigma,
+                                io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream);
+}
+
+int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+             void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+    return step_impl(io, B, M, H, V, p, nullptr, workspace, workspace_bytes, status_dev, cuda_stream);
+}
+
+int psd_step_dag(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
+                 const psd_dag_t* g, void* workspace, size_t workspace_bytes, int32_t* status_dev,
+                 void* cuda_stream) {
+    if (!g) return PSD_ERR_NULL;
+    return step_impl(io, B, M, H, V, p, g, workspace, workspace_bytes, status_dev, cuda_stream);
 }
 
 // Device staging layout of psd_step_host, in order; every piece 256-byte aligned.

@@ -84,8 +84,11 @@ inline CompactSpace carve_compact(void* workspace, int n_rows, int H, int V) {
 }
 
 // combine.cu: merge n_split partial triples per row.
+// pos: NULL, or for every output row the column that holds its partials (-1: the row was not scored
+// and its outputs are left alone).
 int launch_combine(Partials part, int n_split, int n_rows,
-                   int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st);
+                   int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st,
+                   const int32_t* pos = nullptr);
 
 // policy.cu
 int launch_select(const float* conf, const int32_t* tok, const int32_t* node, int n_nodes,

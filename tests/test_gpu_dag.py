@@ -189,3 +189,44 @@ def test_argument_errors():
     with pytest.raises(psd.PsdError) as e:
         psd.psd_verify_accept_dag(x, x.float(), x, x, x, pg, g, x, x, x, x, x)
     assert e.value.code == psd.PSD_ERR_POLICY
+
+
+def test_step_dag_equals_its_stages():
+    """psd_step_dag against the same stages called one by one (merge included), on evolving drafts."""
+    cfg = gen.Config("dagstep", B=6, H=128, V=1500, M=32, D=1, frac=0.8, tau=0.6, k_min=1, k_max=5, seed=33)
+    ranks = GRAPHS["calibrated_like"]
+    K = len(ranks)
+    g = psd.psd_dag_init(ranks)
+    B, M, H, V = cfg.B, cfg.M, cfg.H, cfg.V
+    W = gen.weights(cfg)
+    table, *_ = gen.table_body(cfg, W)
+    w_dev, t_dev = bf16_dev(W), bf16_dev(table.reshape(-1, H))
+    user = psd.table_body_user(t_dev.view(B, M, 3, H), B)
+    tau = f32(cfg.tau)
+    po = oracle.Policy(tau=tau, k_min=1, k_max=5, depth=1, mask_id=cfg.mask_id)
+    pg = psd.policy(tau=tau, k_min=1, k_max=5, depth=1, mask_id=cfg.mask_id)
+    hidden = torch.zeros(B * K * M, H, dtype=torch.bfloat16, device="cuda")
+    buf = psd.StepBuffers.allocate(B, M, K, H, hidden, w_dev, "cuda")
+    buf.tokens.fill_(cfg.mask_id)
+    buf.mask.fill_(1)
+    buf.sigma.fill_(-1)
+    buf.draft_tokens.fill_(cfg.mask_id)
+    buf.draft_mask.fill_(1)
+    ws = torch.empty(psd.psd_workspace_bytes(B * K * M, H, V), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for step in range(5):
+        before = {k: np_(getattr(buf, k)) for k in ("sigma", "draft_tokens", "draft_mask")}
+        psd.psd_table_body(user, buf.draft_mask.view(B * K, M), hidden)
+        psd.psd_step_dag(buf, pg, g, ws, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        tokV, confV = np_(buf.tokV), np_(buf.confV)
+        tokens, mask, ks, ns, nc, _ = oracle.verify_accept_dag(tokV, confV, before["sigma"], before["draft_tokens"],
+                                                               before["draft_mask"], po, ranks)
+        rows = np.arange(B)
+        tokens, mask, sel, n_sel, sel_pos = oracle.select_unmask(confV[rows, ks], tokV[rows, ks], tokens, mask, po)
+        sigma, n_fill, dt, dm = oracle.build_drafts_dag(confV[rows, ks], tokV[rows, ks], tokens, mask, po, ranks)
+        want = dict(k_star=ks, n_spec_accepted=ns, n_committed=nc, tokens=tokens, mask=mask, sel=sel, n_sel=n_sel,
+                    sel_pos=sel_pos, sigma=sigma, n_fill=n_fill, draft_tokens=dt, draft_mask=dm)
+        for k, v in want.items():
+            assert np.array_equal(v, np_(getattr(buf, k))), f"step {step}: {k}"

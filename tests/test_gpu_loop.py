@@ -26,8 +26,12 @@ pytestmark = pytest.mark.gpu
 class Loop:
     """Device buffers of one psd_decode_blocks problem plus the oracle's view of the same table."""
 
-    def __init__(self, cfg, max_iterations=None):
-        self.cfg = cfg
+    def __init__(self, cfg, max_iterations=None, ranks=None):
+        if ranks is not None:                       # the drafts are the nodes of a graph
+            from dataclasses import replace
+            cfg = replace(cfg, D=len(ranks))
+        self.cfg, self.ranks = cfg, ranks
+        self.dag = psd.psd_dag_init(ranks) if ranks is not None else None
         B, M, D, H, V = cfg.B, cfg.M, cfg.D, cfg.H, cfg.V
         self.W = gen.weights(cfg)
         self.table, self.token, self.present, _ = gen.table_body(cfg, self.W)
@@ -62,7 +66,7 @@ class Loop:
         user = psd.table_body_user(self.table_dev.view(self.cfg.B, self.cfg.M, 3, self.cfg.H), self.cfg.B)
         stats = psd.psd_decode_blocks(psd.table_body_address(), ctypes.addressof(user), self.buf, self.pg, order,
                                       self.max_it, self.scratch, self.ws, self.status, self.passes, self.done,
-                                      self.trace)
+                                      self.trace, dag=self.dag)
         torch.cuda.synchronize()
         assert int(self.status.item()) == 0
         return stats
@@ -121,7 +125,7 @@ class Loop:
             return self.tok_o[rows], self.conf_o[rows]
 
         fn = oracle.decode_block if order == psd.ORDER_TWO_PASSES else oracle.decode_block_one_pass
-        return fn(model, M, self.po), clear[0]
+        return fn(model, M, self.po, node_ranks=self.ranks), clear[0]
 
     def compare(self, order, stats):
         cfg = self.cfg
@@ -167,6 +171,23 @@ def test_loop_matches_oracle(name, order):
     if loop.cfg.D > 1:
         assert max(k_stars) > 0                      # some speculation was accepted
         assert stats.iterations < loop.cfg.M         # fewer iterations than slots
+
+
+GRAPH = [set(), {0}, {0, 1}, {1}, {0, 2}, {0, 1, 2}, {0, 1, 2, 3}, {2, 3}, {0, 1, 2, 3, 4, 5}]
+
+
+@pytest.mark.parametrize("compact", [0, 2])
+@pytest.mark.parametrize("order", [psd.ORDER_TWO_PASSES, psd.ORDER_ONE_PASS])
+def test_loop_over_a_draft_graph(order, compact):
+    """Algorithm 1 with a multi-parent draft graph in place of the chain, against the oracle's loop."""
+    loop = Loop(CASES["threshold"], ranks=GRAPH)
+    assert psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, compact) == 0
+    try:
+        stats = loop.run_native(order)
+    finally:
+        psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, 0)
+    set_aside, _, k_stars = loop.compare(order, stats)
+    assert set_aside <= loop.cfg.B // 2 and max(k_stars) > 0 and stats.iterations < loop.cfg.M
 
 
 @pytest.mark.parametrize("name", ["threshold", "long_block"])
