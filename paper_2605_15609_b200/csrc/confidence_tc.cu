@@ -226,13 +226,8 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 
 int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
                           int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(confidence_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) !=
-            cudaSuccess)
-            return PSD_ERR_CUDA;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> smem_set{0};
+    if (!ensure_dynamic_smem(confidence_tc_kernel, SMEM_BYTES, smem_set)) return PSD_ERR_CUDA;
     const int sms = sm_count();
     TileGeometry g = choose_geometry(n_rows, V, sms, max_splits(V), BLOCK_M, 16);
     g.carry = g.n_mt == 1 ? 1 : 0;

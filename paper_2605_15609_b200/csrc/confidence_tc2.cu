@@ -316,13 +316,8 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
 int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
                           int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(confidence_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES) !=
-            cudaSuccess)
-            return PSD_ERR_CUDA;
-        attr_set = true;
-    }
+    static std::atomic<unsigned long long> smem_set{0};
+    if (!ensure_dynamic_smem(confidence_tc2_kernel, SMEM2_BYTES, smem_set)) return PSD_ERR_CUDA;
     const int pairs_max = sm_count() / 2;
     TileGeometry g = choose_geometry(n_rows, V, pairs_max, max_splits(V), 2 * BLOCK_M, 32);
     choose_order(g, n_rows, H, V, 2 * BLOCK_M, band_bytes(), tile_order());

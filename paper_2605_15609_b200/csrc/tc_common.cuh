@@ -2,6 +2,7 @@
 // versions of the fused LM-head + confidence kernel): mbarrier, TMA and tcgen05 wrappers, the
 // running (max, sum-exp, argmax) fold, tensor-map construction.  Everything is internal linkage.
 #pragma once
+#include <atomic>
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include "psd_internal.cuh"
@@ -279,14 +280,28 @@ bool make_map(CUtensorMap* m, const void* base, int rows, int H, int box_rows) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// SM count of the current device (looked up once per device).
 int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
-        return v;
-    }();
-    return n;
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int v = cached[dev].load(std::memory_order_relaxed);
+    if (v > 0) return v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+    cached[dev].store(v, std::memory_order_relaxed);
+    return v;
+}
+
+// The opt-in to more than 48 KB of dynamic shared memory is a per-device property of a kernel: set it
+// the first time the kernel is launched on each device.
+template <typename Kernel>
+bool ensure_dynamic_smem(Kernel kernel, int bytes, std::atomic<unsigned long long>& done_mask) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if ((done_mask.load(std::memory_order_acquire) >> dev) & 1ull) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    done_mask.fetch_or(1ull << dev, std::memory_order_release);
+    return true;
 }
 
 // Chooses how many vocabulary tiles to cut: every tile at most 256 wide, and the tile count such
