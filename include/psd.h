@@ -415,10 +415,11 @@ int psd_table_body(void* user, const int32_t* tokens, const int32_t* mask, int32
 /*
  * Which kernel psd_confidence uses.  Process-wide; returns the previous value, or PSD_ERR_SHAPE for
  * an unknown value.
- *   0  (default) and 2: the tcgen05/TMA kernel, one CTA per tile of 128 rows
+ *   0  (default) the tcgen05/TMA kernels, chosen by size: pairs of CTAs on one tile of 256 rows
+ *      (cta_group::2) for 129..256 rows, one CTA per tile of 128 rows otherwise
  *   1  a plain CUDA-core kernel kept for cross-checking
- *   3  the tcgen05/TMA kernel that runs pairs of CTAs on tiles of 256 rows (cta_group::2); same
- *      results up to summation order, measured slower under the board's power cap
+ *   2  always the single-CTA tcgen05 kernel;  3  always the CTA-pair tcgen05 kernel (same results up
+ *      to summation order)
  */
 int psd_set_confidence_impl(int impl);
 

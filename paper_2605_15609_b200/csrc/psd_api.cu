@@ -39,7 +39,10 @@ int tile_order() { return g_tile_order.load(std::memory_order_relaxed); }
 int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
                          int32_t* status_dev, cudaStream_t st, const int32_t* n_rows_dev) {
     const int impl = g_conf_impl.load(std::memory_order_relaxed);
-    const bool pairs = impl == 3;   // the single-CTA kernel measured faster at every size (see confidence_tc2.cu)
+    // Default choice by measurement (V = 126464, H = 4096): at 129..256 rows one CTA pair covers both row
+    // tiles and fetches every W tile once (258-265 us against 276-282 us); at 128 rows and below, and
+    // from 257 rows up, the single-CTA kernel is faster or equal (see confidence_tc2.cu).
+    const bool pairs = impl == 3 || (impl == 0 && n_rows > 128 && n_rows <= 256);
     return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st)
                  : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st);
 }
