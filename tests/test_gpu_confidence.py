@@ -147,3 +147,34 @@ def test_full_size_configs_sampled_rows(name):
     strong = planted & (wl.scale[:, :, 1:].transpose(0, 2, 1).reshape(-1) >= 4.0)
     want = wl.token[:, :, 1:].transpose(0, 2, 1).reshape(-1)
     assert (tok_g[strong] == want[strong]).mean() > 0.95
+
+
+@pytest.mark.parametrize("impl", [2, 3])
+@pytest.mark.parametrize("order,band_bytes", [(1, 0), (1, 200_000), (2, 70_000), (2, 300_000), (0, 36 << 20)])
+def test_tile_orders_and_ragged_bands(order, band_bytes, impl):
+    """Every tile order (bands of vocabulary tiles, bands of row tiles, band sizes that leave a shorter last
+    band) must visit each (row tile, vocabulary tile) exactly once: results equal the oracle's."""
+    R, H, V = 1500, 128, 3001
+    hid, W = _rand_inputs(77, R, H, V)
+    tok_o, conf_o, lse_o, gap_o = oracle.confidence(hid, W)
+    assert psd.psd_set_tuning(psd.PSD_TUNE_TILE_ORDER, order) == 0
+    assert psd.psd_set_tuning(psd.PSD_TUNE_BAND_BYTES, band_bytes) == 0
+    try:
+        tok_g, conf_g, lse_g = gpu_confidence(bf16_dev(hid), bf16_dev(W), impl=impl)
+    finally:
+        psd.psd_set_tuning(psd.PSD_TUNE_TILE_ORDER, 0)
+        psd.psd_set_tuning(psd.PSD_TUNE_BAND_BYTES, 36 << 20)
+    check_confidence(tok_g, conf_g, lse_g, tok_o, conf_o, lse_o, gap_o)
+
+
+def test_many_rows_small_problem():
+    # 547 row tiles: more tiles than one pass of the persistent grid many times over
+    R, H, V = 70000, 64, 300
+    rng = np.random.default_rng(5)
+    W = gen.bf16_bits(rng.normal(scale=0.3, size=(V, H)).astype(np.float32))
+    hid = gen.bf16_bits(rng.normal(size=(R, H)).astype(np.float32))
+    tok_g, conf_g, lse_g = gpu_confidence(bf16_dev(hid), bf16_dev(W))
+    rows = np.unique(np.concatenate([[0, 127, 128, R - 1, R - 113], rng.integers(0, R, size=300)]))
+    tok_o, conf_o, lse_o, gap_o = oracle.confidence(hid[rows], W)
+    check_confidence(tok_g[rows], conf_g[rows], lse_g[rows], tok_o, conf_o, lse_o, gap_o)
+    assert (tok_g >= 0).all() and (tok_g < V).all() and (conf_g > 1.0 / V - 1e-6).all() and (conf_g <= 1.0 + 1e-6).all()
