@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel, from the ncu captures
 # summarised under profiles/ (None where no capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"single_request": 1.0407e9, "batched_serving": 2.192e9}
+NCU_TRAFFIC_BYTES = {"single_request": 1.0406e9, "batched_serving": 2.193e9}
 
 
 def load_peaks():
