@@ -455,7 +455,7 @@ def main():
                     help="time the whole decoding loop (psd_decode_blocks) instead of one step; an extra "
                          "measurement, not the headline metric")
     ap.add_argument("--compact", action="store_true",
-                    help="with --loop one_pass: score only the rows of slots still masked in their draft")
+                    help="with --loop: score only the rows of slots that are still masked")
     ap.add_argument("--profile-only", action="store_true",
                     help="for runs under a profiler: device-resident steps only (no instrumented pass, no "
                          "end-to-end pass, no CPU baseline); the printed line is not a benchmark result")

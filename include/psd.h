@@ -122,6 +122,20 @@ int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t
                    int32_t* status_dev, void* cuda_stream);
 
 /*
+ * psd_confidence_masked — psd_confidence on the rows whose row_mask is non-zero, without the host
+ * knowing how many there are (Sec. 3.2 Stage 3 needs predictions only at "each masked position").
+ * row_mask [n_rows] int32, device: typically the mask of the sequences themselves ([B, M] or
+ * [B, D, M] flattened).  Outputs of flagged rows are written at the rows' own places; outputs of the
+ * other rows are left untouched.  No host synchronisation: the rows are listed and copied into a dense
+ * buffer on the device, and the fused kernel reads their number from device memory.
+ * workspace >= psd_compact_workspace_bytes(n_rows, H, V).  Other arguments as for psd_confidence.
+ */
+int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_mask,
+                          int32_t n_rows, int32_t H, int32_t V,
+                          int32_t* out_token, float* out_conf, float* out_lse,
+                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+
+/*
  * psd_select_unmask — the transfer policy T = pi(x, c) and the state update of Eq. (1).
  * (Sec. 3.2 Stage 1; App. B.2 for the threshold rule.)
  *
@@ -444,6 +458,8 @@ int psd_set_confidence_impl(int impl);
  *                        psd_compact_workspace_bytes, and entries of tokV / confV that belong to
  *                        committed slots are left as they were (no stage reads them) */
 #define PSD_TUNE_COMPACT_ROWS 4
+/* 1 if PSD_TUNE_COMPACT_ROWS makes a batch of n_rows rows take the compacted path, else 0. */
+int psd_compact_rows_enabled(int32_t n_rows);
 int psd_set_tuning(int knob, int value);
 
 /*

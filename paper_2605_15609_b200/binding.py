@@ -78,6 +78,10 @@ def _load() -> ctypes.CDLL:
     lib.psd_compact_workspace_bytes.argtypes = [_i32, _i32, _i32]
     lib.psd_confidence.restype = ctypes.c_int
     lib.psd_confidence.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    lib.psd_confidence_masked.restype = ctypes.c_int
+    lib.psd_confidence_masked.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    lib.psd_compact_rows_enabled.restype = ctypes.c_int
+    lib.psd_compact_rows_enabled.argtypes = [_i32]
     lib.psd_confidence_static.restype = ctypes.c_int
     lib.psd_confidence_static.argtypes = [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
     lib.psd_select_unmask.restype = ctypes.c_int
@@ -203,6 +207,21 @@ def psd_confidence(hidden, w_lm, out_token, out_conf, out_lse=None, workspace=No
     _check(LIB.psd_confidence(_ptr(hidden), _ptr(w_lm), _ptr(row_ids), n_rows, H, V, _ptr(out_token),
                               _ptr(out_conf), _ptr(out_lse), _ptr(workspace), ws_bytes, _ptr(status),
                               _stream(stream)), "psd_confidence")
+
+
+def psd_confidence_masked(hidden, w_lm, row_mask, out_token, out_conf, out_lse=None, workspace=None, status=None,
+                          stream=None):
+    """psd_confidence on the rows whose ``row_mask`` (int32, device, one entry per row of ``hidden``) is
+    non-zero; the other rows' outputs are left untouched.  No host synchronisation."""
+    n_rows, H = hidden.shape
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(LIB.psd_confidence_masked(_ptr(hidden), _ptr(w_lm), _ptr(row_mask), n_rows, H, w_lm.shape[0],
+                                     _ptr(out_token), _ptr(out_conf), _ptr(out_lse), _ptr(workspace), ws_bytes,
+                                     _ptr(status), _stream(stream)), "psd_confidence_masked")
+
+
+def psd_compact_rows_enabled(n_rows: int) -> int:
+    return int(LIB.psd_compact_rows_enabled(int(n_rows)))
 
 
 PSD_STATIC_SCRATCH_BYTES = 4 << 20

@@ -196,9 +196,12 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
         } else {
             // Algorithm 1 as printed.  Stage 1: one pass on the current state, policy, Eq. (1).
             if ((e = body(user, io->tokens, io->mask, B, M, hidden, cuda_stream))) return e;
-            if ((e = psd_confidence(hidden, io->w_lm_bf16, nullptr, B * M, H, V, tok1, conf1, nullptr, workspace,
-                                    workspace_bytes, status_dev, cuda_stream)))
-                return e;
+            e = psd_compact_rows_enabled(B * M)
+                    ? psd_confidence_masked(hidden, io->w_lm_bf16, io->mask, B * M, H, V, tok1, conf1, nullptr,
+                                            workspace, workspace_bytes, status_dev, cuda_stream)
+                    : psd_confidence(hidden, io->w_lm_bf16, nullptr, B * M, H, V, tok1, conf1, nullptr, workspace,
+                                     workspace_bytes, status_dev, cuda_stream);
+            if (e) return e;
             if ((e = psd_select_unmask(conf1, tok1, nullptr, 1, io->tokens, io->mask, B, M, p, io->sel, io->n_sel,
                                        io->sel_pos, cuda_stream)))
                 return e;
@@ -216,9 +219,13 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
                                          io->n_fill, io->draft_tokens, io->draft_mask, cuda_stream);
                 if (e) return e;
                 if ((e = body(user, io->draft_tokens, io->draft_mask, B * D, M, hidden, cuda_stream))) return e;
-                if ((e = psd_confidence(hidden, io->w_lm_bf16, nullptr, B * D * M, H, V, io->tokV, io->confV, nullptr,
-                                        workspace, workspace_bytes, status_dev, cuda_stream)))
-                    return e;
+                e = psd_compact_rows_enabled(B * D * M)
+                        ? psd_confidence_masked(hidden, io->w_lm_bf16, io->draft_mask, B * D * M, H, V, io->tokV,
+                                                io->confV, nullptr, workspace, workspace_bytes, status_dev,
+                                                cuda_stream)
+                        : psd_confidence(hidden, io->w_lm_bf16, nullptr, B * D * M, H, V, io->tokV, io->confV,
+                                         nullptr, workspace, workspace_bytes, status_dev, cuda_stream);
+                if (e) return e;
                 e = g ? psd_verify_accept_dag(io->tokV, io->confV, io->sigma, io->draft_tokens, io->draft_mask, B, M,
                                               p, g, io->tokens, io->mask, io->k_star, io->n_spec_accepted,
                                               io->n_committed, nullptr, cuda_stream)

@@ -77,6 +77,11 @@ size_t psd_compact_workspace_bytes(int32_t n_rows, int32_t H, int32_t V) {
     return partial_bytes(n_rows, V) + compact_extra_bytes(n_rows, H);
 }
 
+int psd_compact_rows_enabled(int32_t n_rows) {
+    const int mode = g_compact.load(std::memory_order_relaxed);
+    return (mode == 2 || (mode == 1 && n_rows > 128)) ? 1 : 0;
+}
+
 int psd_set_confidence_impl(int impl) {
     if (impl < 0 || impl > 3) return PSD_ERR_SHAPE;
     return g_conf_impl.exchange(impl);
@@ -147,6 +152,37 @@ int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t
     return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st);
 }
 
+int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_mask,
+                          int32_t n_rows, int32_t H, int32_t V,
+                          int32_t* out_token, float* out_conf, float* out_lse,
+                          void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+    if (!hidden_bf16 || !w_lm_bf16 || !row_mask || !out_token || !out_conf || !workspace) return PSD_ERR_NULL;
+    if (!conf_shape_ok(n_rows, H, V)) return PSD_ERR_SHAPE;
+    if (!aligned(hidden_bf16, 16) || !aligned(w_lm_bf16, 16) || !aligned(workspace, 256) || !aligned(row_mask, 4) ||
+        !aligned(out_token, 4) || !aligned(out_conf, 4) || !aligned(out_lse, 4) || !aligned(status_dev, 4))
+        return PSD_ERR_ALIGN;
+    if (workspace_bytes < psd_compact_workspace_bytes(n_rows, H, V)) return PSD_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    Partials part = carve_partials(workspace, n_rows, V);
+    CompactSpace cs = carve_compact(workspace, n_rows, H, V);
+    // list the flagged rows, copy them into a dense buffer, score as many rows as the device-side count
+    // says, and merge every flagged row's partials back to the row's own place
+    if (int e = launch_list_rows(row_mask, n_rows, cs.row_ids, cs.pos, cs.count, st)) return e;
+    if (int e = launch_gather_rows(hidden_bf16, cs.row_ids, cs.count, 0, n_rows, H, cs.hidden, st)) return e;
+    const bool timed = t_ev_start && t_ev_stop;
+    if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
+    int n_split = g_conf_impl.load() == 1
+                      ? launch_confidence_simt(cs.hidden, w_lm_bf16, n_rows, H, V, part, st)
+                      : launch_confidence_tc(cs.hidden, w_lm_bf16, n_rows, H, V, part, status_dev, st, cs.count);
+    if (timed) {
+        cudaError_t e = cudaEventRecord(t_ev_stop, st);
+        t_ev_start = t_ev_stop = nullptr;
+        if (e != cudaSuccess) return PSD_ERR_CUDA;
+    }
+    if (n_split < 0) return n_split;
+    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, cs.pos);
+}
+
 int psd_select_unmask(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
                       int32_t* tokens, int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
                       int32_t* sel, int32_t* n_sel, int32_t* sel_pos, void* cuda_stream) {
@@ -209,8 +245,7 @@ static int step_impl(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, i
     if (!aligned(io->hidden_bf16, 16) || !aligned(io->w_lm_bf16, 16) || !aligned(workspace, 256) ||
         !aligned(status_dev, 4))
         return PSD_ERR_ALIGN;
-    const int compact_mode = g_compact.load(std::memory_order_relaxed);
-    const bool compact = compact_mode == 2 || (compact_mode == 1 && n_rows > 128);
+    const bool compact = psd_compact_rows_enabled(n_rows) != 0;
     if (workspace_bytes < (compact ? psd_compact_workspace_bytes(n_rows, H, V) : psd_workspace_bytes(n_rows, H, V)))
         return PSD_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);

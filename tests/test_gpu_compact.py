@@ -126,3 +126,31 @@ def test_small_workspace_is_rejected(compaction):
     compaction(0)
     psd.psd_step(buf, pg, ws, None)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("impl", [0, 1, 3])
+@pytest.mark.parametrize("R,frac", [(1, 1.0), (130, 0.5), (300, 0.1), (300, 0.0), (700, 0.9)])
+def test_confidence_masked(R, frac, impl):
+    rng = np.random.default_rng(R + int(frac * 10))
+    H, V = 128, 2500
+    W = gen.bf16_bits(rng.normal(scale=0.05, size=(V, H)).astype(np.float32))
+    hid = gen.bf16_bits((rng.normal(size=(R, H)) * rng.uniform(0.5, 6.0, size=(R, 1))).astype(np.float32))
+    flags = (rng.random(R) < frac).astype(np.int32)
+    tok = torch.full((R,), -7, dtype=torch.int32, device="cuda")
+    conf = torch.full((R,), -7.0, dtype=torch.float32, device="cuda")
+    lse = torch.full((R,), -7.0, dtype=torch.float32, device="cuda")
+    ws = torch.empty(psd.psd_compact_workspace_bytes(R, H, V), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    prev = psd.psd_set_confidence_impl(impl)
+    try:
+        psd.psd_confidence_masked(bf16_dev(hid), bf16_dev(W), dev(flags), tok, conf, lse, ws, status)
+        torch.cuda.synchronize()
+    finally:
+        psd.psd_set_confidence_impl(prev)
+    assert int(status.item()) == 0
+    tok, conf, lse = np_(tok), np_(conf), np_(lse)
+    on = flags != 0
+    assert (tok[~on] == -7).all() and (conf[~on] == -7.0).all() and (lse[~on] == -7.0).all()
+    if on.any():
+        tok_o, conf_o, lse_o, gap_o = oracle.confidence(hid[on], W)
+        check_confidence(tok[on], conf[on], lse[on], tok_o, conf_o, lse_o, gap_o)

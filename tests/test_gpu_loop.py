@@ -190,16 +190,17 @@ def test_loop_over_a_draft_graph(order, compact):
     assert set_aside <= loop.cfg.B // 2 and max(k_stars) > 0 and stats.iterations < loop.cfg.M
 
 
+@pytest.mark.parametrize("order", [psd.ORDER_TWO_PASSES, psd.ORDER_ONE_PASS])
 @pytest.mark.parametrize("name", ["threshold", "long_block"])
-def test_loop_with_row_compaction(name):
-    """The one-pass loop with psd_step scoring only masked rows: same parity bar."""
+def test_loop_with_row_compaction(name, order):
+    """The loop scoring only masked rows (psd_step's compaction, psd_confidence_masked): same parity bar."""
     loop = Loop(CASES[name])
     assert psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, 2) == 0
     try:
-        stats = loop.run_native(psd.ORDER_ONE_PASS)
+        stats = loop.run_native(order)
     finally:
         psd.psd_set_tuning(psd.PSD_TUNE_COMPACT_ROWS, 0)
-    set_aside, _, k_stars = loop.compare(psd.ORDER_ONE_PASS, stats)
+    set_aside, _, k_stars = loop.compare(order, stats)
     assert set_aside <= loop.cfg.B // 2 and max(k_stars) > 0
 
 
