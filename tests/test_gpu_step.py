@@ -155,3 +155,30 @@ def test_psd_step_host_matches_device_step(name, one_block):
     assert psd.psd_step_host(hb, pg, staging) == 0
     for k in STEP_INT_OUTPUTS + ("tokV", "confV"):
         assert np.array_equal(getattr(hb, k).numpy(), want[k]), k
+
+
+def test_psd_step_can_be_captured_in_a_cuda_graph():
+    """The step is two launches with by-value tensor maps and no host synchronisation, so a stream
+    capture of it replays to the same outputs as direct calls."""
+    cfg, wl, w_dev = _workload("tiny")
+    po, pg = policies(cfg)
+    _, chain = gpu_prologue(cfg, bf16_dev(wl.hidden_stage1), w_dev, pg)
+    hv = bf16_dev(wl.hidden_verify)
+    ws = torch.empty(psd.psd_workspace_bytes(cfg.rows, cfg.H, cfg.V), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ref = step_buffers_from(chain, cfg, hv, w_dev)
+    for _ in range(3):
+        psd.psd_step(ref, pg, ws, status)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    buf = step_buffers_from(chain, cfg, hv, w_dev)
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            psd.psd_step(buf, pg, ws, status, side)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for k in STEP_INT_OUTPUTS + ("tokV", "confV"):
+        assert torch.equal(getattr(buf, k), getattr(ref, k)), k
