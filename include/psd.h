@@ -105,7 +105,8 @@ size_t psd_compact_workspace_bytes(int32_t n_rows, int32_t H, int32_t V);
  *   hidden_bf16  [n_rows, H] bf16, 16-byte aligned, device
  *   w_lm_bf16    [V, H]      bf16, 16-byte aligned, device
  *   row_ids      NULL, or a device list [n_rows] int32 of the rows of hidden_bf16 to score (a gather list:
- *                output r belongs to hidden row row_ids[r]; hidden_bf16 may then have any number of rows).
+ *                output r belongs to hidden row row_ids[r]; hidden_bf16 may then have any number of rows;
+ *                every id must be a valid row of it, the library does not check).
  *                The workspace must then hold psd_compact_workspace_bytes(n_rows, H, V)
  *   n_rows >= 1;  H >= 64 and a multiple of 64;  1 <= V < 2^31 - 256
  *   out_token    [n_rows] int32;  out_conf [n_rows] fp32;  out_lse [n_rows] fp32 or NULL
