@@ -137,6 +137,28 @@ int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const 
                           void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
 
 /*
+ * ---- The vocabulary split over several GPUs ----------------------------------------------------------
+ * softmax max / argmax over the whole vocabulary is an associative merge of per-range triples
+ * (max logit, sum of exp(logit - max), lowest argmax), the same merge that combines the vocabulary
+ * tiles inside psd_confidence.  A GPU that holds rows [v_offset, v_offset + V_shard) of W computes its
+ * triple per row; the triples of all GPUs (12 bytes per row and GPU) are exchanged by the caller and
+ * merged on every GPU.  (Sec. 3.1 defines x^ and c over the whole vocabulary; the split is this
+ * library's, for LM heads sharded over GPUs.)
+ *
+ * psd_confidence_partial: out_max, out_sumexp [n_rows] fp32, out_arg [n_rows] int32 (GLOBAL vocabulary
+ *   index); other arguments as for psd_confidence with V = V_shard.
+ * psd_merge_partials: max, sumexp, arg are [n_shards, n_rows] (shard-major, e.g. the all-gathered
+ *   outputs of psd_confidence_partial); out_token, out_conf, out_lse as for psd_confidence.  Equal
+ *   maxima keep the lowest global index, so the result does not depend on the number of shards
+ *   beyond the rounding order of the sums.
+ */
+int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, int32_t n_rows, int32_t H,
+                           int32_t V_shard, int32_t v_offset, float* out_max, float* out_sumexp, int32_t* out_arg,
+                           void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
+int psd_merge_partials(const float* max, const float* sumexp, const int32_t* arg, int32_t n_shards, int32_t n_rows,
+                       int32_t* out_token, float* out_conf, float* out_lse, void* cuda_stream);
+
+/*
  * psd_select_unmask — the transfer policy T = pi(x, c) and the state update of Eq. (1).
  * (Sec. 3.2 Stage 1; App. B.2 for the threshold rule.)
  *

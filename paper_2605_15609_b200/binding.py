@@ -82,6 +82,10 @@ def _load() -> ctypes.CDLL:
     lib.psd_confidence_masked.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
     lib.psd_compact_rows_enabled.restype = ctypes.c_int
     lib.psd_compact_rows_enabled.argtypes = [_i32]
+    lib.psd_confidence_partial.restype = ctypes.c_int
+    lib.psd_confidence_partial.argtypes = [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    lib.psd_merge_partials.restype = ctypes.c_int
+    lib.psd_merge_partials.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp]
     lib.psd_confidence_static.restype = ctypes.c_int
     lib.psd_confidence_static.argtypes = [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
     lib.psd_select_unmask.restype = ctypes.c_int
@@ -222,6 +226,23 @@ def psd_confidence_masked(hidden, w_lm, row_mask, out_token, out_conf, out_lse=N
 
 def psd_compact_rows_enabled(n_rows: int) -> int:
     return int(LIB.psd_compact_rows_enabled(int(n_rows)))
+
+
+def psd_confidence_partial(hidden, w_shard, v_offset, out_max, out_sumexp, out_arg, workspace, status=None,
+                           stream=None):
+    """Per-row (max, sum-exp, global argmax) over the vocabulary rows held in ``w_shard`` [V_shard, H]."""
+    n_rows, H = hidden.shape
+    _check(LIB.psd_confidence_partial(_ptr(hidden), _ptr(w_shard), n_rows, H, w_shard.shape[0], int(v_offset),
+                                      _ptr(out_max), _ptr(out_sumexp), _ptr(out_arg), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _ptr(status), _stream(stream)),
+           "psd_confidence_partial")
+
+
+def psd_merge_partials(max_, sumexp, arg, out_token, out_conf, out_lse=None, stream=None):
+    """Merge [n_shards, n_rows] triples into token / confidence / lse per row."""
+    n_shards, n_rows = max_.shape
+    _check(LIB.psd_merge_partials(_ptr(max_), _ptr(sumexp), _ptr(arg), n_shards, n_rows, _ptr(out_token),
+                                  _ptr(out_conf), _ptr(out_lse), _stream(stream)), "psd_merge_partials")
 
 
 PSD_STATIC_SCRATCH_BYTES = 4 << 20

@@ -36,7 +36,8 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
                                                const int32_t* __restrict__ pa, int n_split, int n_rows,
                                                int row0, int row_end, int g, Triple (*sh)[kCombineRows],
                                                int32_t* __restrict__ out_token, float* __restrict__ out_conf,
-                                               float* __restrict__ out_lse, const int32_t* __restrict__ pos = nullptr) {
+                                               float* __restrict__ out_lse, const int32_t* __restrict__ pos = nullptr,
+                                               float* __restrict__ out_max = nullptr, int32_t arg_offset = 0) {
     const int tx = g & 31, lane = g >> 5;
     const int out_row = row0 + tx;
     // with compacted rows the partials of output row r sit in column pos[r]; -1 = the row was not scored
@@ -72,9 +73,16 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
             const Triple y = sh[l][tx];
             if (y.a != INT32_MAX) merge_triple(x, y.m, y.s, y.a);
         }
-        out_token[out_row] = x.a;
-        out_conf[out_row] = 1.0f / x.s;
-        if (out_lse) out_lse[out_row] = x.m + logf(x.s);
+        if (out_max) {
+            // the merged triple itself (one shard of the vocabulary): max, sum-exp, argmax as a global index
+            out_max[out_row] = x.m;
+            out_conf[out_row] = x.s;
+            out_token[out_row] = x.a + arg_offset;
+        } else {
+            out_token[out_row] = x.a;
+            out_conf[out_row] = 1.0f / x.s;
+            if (out_lse) out_lse[out_row] = x.m + logf(x.s);
+        }
     }
     __syncthreads();
 }

@@ -183,6 +183,36 @@ int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const 
     return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, cs.pos);
 }
 
+int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, int32_t n_rows, int32_t H,
+                           int32_t V_shard, int32_t v_offset, float* out_max, float* out_sumexp, int32_t* out_arg,
+                           void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream) {
+    if (!hidden_bf16 || !w_shard_bf16 || !out_max || !out_sumexp || !out_arg || !workspace) return PSD_ERR_NULL;
+    if (!conf_shape_ok(n_rows, H, V_shard) || v_offset < 0 || (long long)v_offset + V_shard > 2147483647ll - 256)
+        return PSD_ERR_SHAPE;
+    if (!aligned(hidden_bf16, 16) || !aligned(w_shard_bf16, 16) || !aligned(workspace, 256) || !aligned(out_max, 4) ||
+        !aligned(out_sumexp, 4) || !aligned(out_arg, 4) || !aligned(status_dev, 4))
+        return PSD_ERR_ALIGN;
+    if (workspace_bytes < psd_workspace_bytes(n_rows, H, V_shard)) return PSD_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+    Partials part = carve_partials(workspace, n_rows, V_shard);
+    int n_split = g_conf_impl.load() == 1
+                      ? launch_confidence_simt(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, st)
+                      : launch_confidence_tc(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, status_dev, st);
+    if (n_split < 0) return n_split;
+    return launch_combine(part, n_split, n_rows, out_arg, out_sumexp, nullptr, st, nullptr, out_max, v_offset);
+}
+
+int psd_merge_partials(const float* max, const float* sumexp, const int32_t* arg, int32_t n_shards, int32_t n_rows,
+                       int32_t* out_token, float* out_conf, float* out_lse, void* cuda_stream) {
+    if (!max || !sumexp || !arg || !out_token || !out_conf) return PSD_ERR_NULL;
+    if (n_shards < 1 || n_rows < 1) return PSD_ERR_SHAPE;
+    Partials part;
+    part.m = const_cast<float*>(max);
+    part.s = const_cast<float*>(sumexp);
+    part.a = const_cast<int32_t*>(arg);
+    return launch_combine(part, n_shards, n_rows, out_token, out_conf, out_lse, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
 int psd_select_unmask(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
                       int32_t* tokens, int32_t* mask, int32_t B, int32_t M, psd_policy_t p,
                       int32_t* sel, int32_t* n_sel, int32_t* sel_pos, void* cuda_stream) {

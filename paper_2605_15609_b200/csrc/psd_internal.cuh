@@ -88,7 +88,9 @@ inline CompactSpace carve_compact(void* workspace, int n_rows, int H, int V) {
 // and its outputs are left alone).
 int launch_combine(Partials part, int n_split, int n_rows,
                    int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st,
-                   const int32_t* pos = nullptr);
+                   const int32_t* pos = nullptr, float* out_max = nullptr, int32_t arg_offset = 0);
+// With out_max the kernel writes the merged triple instead: out_max = max, out_conf = sum-exp,
+// out_token = argmax + arg_offset.
 
 // policy.cu
 int launch_select(const float* conf, const int32_t* tok, const int32_t* node, int n_nodes,
