@@ -450,6 +450,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", default="single_request",
                     help="workload: tiny, single_request, class_7b, batched_serving, deep_sweep[_D1|_D2|_D4]")
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="override the workload's number of blocks B (rows = B*D*M), e.g. to sweep row counts "
+                         "across the HBM/tensor ridge; the printed config names the override")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loop", default=None, choices=["one_pass", "two_passes"],
                     help="time the whole decoding loop (psd_decode_blocks) instead of one step; an extra "
@@ -468,6 +471,8 @@ def main():
         cfg = gen.with_depth(gen.CONFIGS["deep_sweep"], int(name.rsplit("D", 1)[1]))
     else:
         cfg = gen.CONFIGS[name]
+    if args.blocks > 0:
+        cfg = replace(cfg, B=args.blocks, name=f"{cfg.name}_B{args.blocks}")
     if args.impl == "reference":
         return run_reference(args, cfg)
     if args.loop:
