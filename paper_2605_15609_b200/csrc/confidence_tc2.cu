@@ -271,6 +271,8 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const uint32_t acc_empty0 = map_to_cta(smem_u32(&acc_empty_bar[0]), 0);   // the leader's acc_empty[0]
         int it = 0;
         bool ok = true;
+        float run_m = -INFINITY, run_s = 0.f;
+        int run_a = 0;
         for (int t = pair_id; t < n_tiles && ok; t += n_pairs, ++it) {
             int m_tile, v_tile, v0, ncols;
             decode_tile(geo, t, m_tile, v_tile, v0, ncols);
@@ -278,8 +280,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, abort_flag, status_dev)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
-            float run_m = -INFINITY, run_s = 0.f;
-            int run_a = 0;
+            if (!geo.carry) { run_m = -INFINITY; run_s = 0.f; run_a = 0; }
             const bool ragged = v0 + ncols > V;
             for (int c = 0; c < ncols; c += 32) {
                 float x[32];
@@ -294,9 +295,12 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty0 + (uint32_t)acc * 8);
+            // One row tile (at most 256 rows): a pair's tiles come in ascending vocabulary order, so each
+            // thread carries one running triple across them and writes it once, to split slot pair_id.
+            const bool last_of_pair = t + n_pairs >= n_tiles;
             const int row = m_tile * 256 + (int)rank * BLOCK_M + row_in_tile;
-            if (row < n_rows_act) {
-                const size_t o = (size_t)v_tile * n_rows + row;
+            if (row < n_rows_act && (!geo.carry || last_of_pair)) {
+                const size_t o = (size_t)(geo.carry ? pair_id : v_tile) * n_rows + row;
                 pm[o] = run_m;
                 ps[o] = run_s;
                 pa[o] = run_a;
@@ -322,7 +326,8 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     if (!ensure_dynamic_smem(confidence_tc2_kernel, SMEM2_BYTES, smem_set)) return PSD_ERR_CUDA;
     const int pairs_max = sm_count() / 2;
     TileGeometry g = choose_geometry(n_rows, V, pairs_max, max_splits(V), 2 * BLOCK_M, 32);
-    choose_order(g, n_rows, H, V, 2 * BLOCK_M, band_bytes(), tile_order());
+    g.carry = g.n_mt == 1 ? 1 : 0;
+    choose_order(g, n_rows, H, V, 2 * BLOCK_M, band_bytes(), g.carry ? 1 : tile_order());
     const int wide_half = (g.rem ? g.base_units + 1 : g.base_units) * 16;      // half of unit 32
     const int narrow_half = g.base_units > 0 ? g.base_units * 16 : wide_half;
     CUtensorMap map_a, map_bw, map_bn;
@@ -338,14 +343,15 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 0;   // plain stream order (see the single-CTA launcher)
+    // early start only for one row tile, as in the single-CTA launcher
+    attr[0].val.programmaticStreamSerializationAllowed = (pdl_enabled() && g.n_mt == 1) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc2_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
                                        part.s, part.a, status_dev, n_rows_dev);
     count_launch();
     if (e != cudaSuccess) return PSD_ERR_CUDA;
-    return g.n_vt;
+    return g.carry ? pairs : g.n_vt;   // number of split slots written per row
 }
 
 }  // namespace psd
