@@ -286,8 +286,8 @@ int psd_step(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V
              void* workspace, size_t workspace_bytes, int32_t* status_dev, void* cuda_stream);
 
 /*
- * Bytes of device staging that psd_step_host needs (inputs, outputs and psd_confidence's
- * scratch).  Returns 0 for invalid sizes.
+ * Bytes of device staging that psd_step_host needs (inputs, outputs and the step's scratch, sized so
+ * that PSD_TUNE_COMPACT_ROWS may be on).  Returns 0 for invalid sizes.
  */
 size_t psd_step_host_bytes(int32_t B, int32_t M, int32_t H, int32_t V, int32_t D);
 

@@ -364,7 +364,7 @@ Staging staging_layout(int B, int M, int H, int V, int D) {
     s.n_sel = take((size_t)B * 4);
     s.sel_pos = take(BM * 4);
     s.status = take(4);
-    s.workspace = take(psd_workspace_bytes((int)R, H, V));
+    s.workspace = take(psd_compact_workspace_bytes((int)R, H, V));   // also enough when row compaction is on
     s.total = o;
     return s;
 }

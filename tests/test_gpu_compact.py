@@ -154,3 +154,23 @@ def test_confidence_masked(R, frac, impl):
     if on.any():
         tok_o, conf_o, lse_o, gap_o = oracle.confidence(hid[on], W)
         check_confidence(tok[on], conf[on], lse[on], tok_o, conf_o, lse_o, gap_o)
+
+
+def test_host_step_with_compaction(compaction):
+    """psd_step_host sizes its staging for the compacted path too."""
+    cfg, wl, w_dev = _workload("medium")
+    po, pg = policies(cfg)
+    _, chain = gpu_prologue(cfg, bf16_dev(wl.hidden_stage1), w_dev, pg)
+    hv_dev = bf16_dev(wl.hidden_verify)
+    ref = step_buffers_from(chain, cfg, hv_dev, w_dev)
+    ws = torch.empty(psd.psd_workspace_bytes(cfg.rows, cfg.H, cfg.V), dtype=torch.uint8, device="cuda")
+    psd.psd_step(ref, pg, ws, None)
+    torch.cuda.synchronize()
+    hb = psd.host_step_buffers(cfg.B, cfg.M, cfg.D, hv_dev.cpu().pin_memory(), w_dev)
+    for k in ("sigma", "n_fill", "draft_tokens", "draft_mask"):
+        getattr(hb, k).copy_(getattr(chain, k))
+    staging = torch.empty(psd.psd_step_host_bytes(cfg.B, cfg.M, cfg.H, cfg.V, cfg.D), dtype=torch.uint8, device="cuda")
+    compaction(2)
+    assert psd.psd_step_host(hb, pg, staging) == 0
+    for k in STEP_INT_OUTPUTS:
+        assert np.array_equal(getattr(hb, k).numpy(), np_(getattr(ref, k))), k
