@@ -288,13 +288,21 @@ def run_ours(args, cfg):
     # ---- device-resident steps: the headline value
     for _ in range(args.warmup):
         psd.psd_step(buf, pg, ws, status, stream)
-    sampler = ClockSampler(physical_gpu_index(info.local_rank))
-    launches0 = psd.psd_launch_count()
-    sampler.start()
-    secs = timed_region(lambda i: psd.psd_step(buf, pg, ws, status, stream), args.steps)
-    sampler.sample()
-    sampler.stop()
-    launches = psd.psd_launch_count() - launches0
+    remeasured = False
+    while True:
+        sampler = ClockSampler(physical_gpu_index(info.local_rank))
+        launches0 = psd.psd_launch_count()
+        sampler.start()
+        secs = timed_region(lambda i: psd.psd_step(buf, pg, ws, status, stream), args.steps)
+        sampler.sample()
+        sampler.stop()
+        launches = psd.psd_launch_count() - launches0
+        # a timed region that saw a hardware or thermal slowdown is taken again, once
+        bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(sampler.summary()["reasons"])
+        if not bad or remeasured:
+            break
+        remeasured = True
+        time.sleep(2.0)
     if int(status.item()) != 0:
         raise RuntimeError("device status: " + psd.status_string(int(status.item())))
     value, secs_max = replicas.aggregate_throughput(float(R) * args.steps, secs, info, device)
@@ -367,7 +375,7 @@ def run_ours(args, cfg):
                        "policy": {"tau": cfg.tau, "k_min": cfg.k_min, "k_max": cfg.k_max, "stride": cfg.stride},
                        "parallelism": f"replicas x{info.world_size}",
                        "l2": f"inputs larger than L2: W is {V * H * 2 / 1e6:.0f} MB and is re-read every step"},
-            "clocks": sampler.summary(),
+            "clocks": dict(sampler.summary(), remeasured=remeasured),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": 1e3 * secs_e2e / n_e2e, "steps": n_e2e},
             "gpu_launches": launches,
