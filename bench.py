@@ -299,7 +299,8 @@ def run_ours(args, cfg):
         launches = psd.psd_launch_count() - launches0
         # a timed region that saw a hardware or thermal slowdown is taken again, once
         bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(sampler.summary()["reasons"])
-        if not bad or remeasured:
+        bad_anywhere = replicas.max_over_ranks(1.0 if bad else 0.0, info, device) > 0   # all ranks decide alike
+        if not bad_anywhere or remeasured:
             break
         remeasured = True
         time.sleep(2.0)
