@@ -31,7 +31,10 @@
 namespace psd {
 namespace {
 
-constexpr int STAGES2 = 6;
+#ifndef PSD_STAGES2
+#define PSD_STAGES2 6
+#endif
+constexpr int STAGES2 = PSD_STAGES2;               // depth of the shared-memory ring (32 KB per stage)
 constexpr int HALF_N = BLOCK_N / 2;                  // widest half tile of W held by one CTA
 constexpr int B2_BYTES = HALF_N * BLOCK_K * 2;       // 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + B2_BYTES;     // 32 KB
