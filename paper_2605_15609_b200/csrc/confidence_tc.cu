@@ -90,9 +90,6 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            // W is read once per row tile: with a single row tile it streams through L2, otherwise the
-            // row tiles that run side by side share it for a short while; hidden is re-read for every
-            // vocabulary tile and should stay resident.
             // One row tile: W streams through L2 once and is marked to leave first; the hidden rows are
             // re-read for every vocabulary tile and stay.  Several row tiles: both operands are re-read
             // from L2 many times within a band, and marking both to stay measured fastest (8192 rows:
