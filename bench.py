@@ -8,6 +8,12 @@ B*D*M rows of the verification batch, then psd_verify_accept, psd_select_unmask 
 psd_build_drafts (psd_step), on one stream.  The metric is masked positions scored and accepted
 per second = B*D*M / t_step.  Rank 0 prints ONE JSON line.
 
+Without --config the line's own result is the largest single-GPU workload (batched_serving: 8192
+rows, bound by the bf16 tensor pipe) and the key "single_request" holds the same measurements of
+the 128-row workload (bound by the one pass over W in HBM), so that one run covers both regimes.
+A timed region is exactly K steps; it is repeated until --min-seconds of device time have passed
+and the median region is reported with the spread.
+
 For N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs an independent
 replica on its own batch: no data-path collective, weak scaling.
 
@@ -36,8 +42,11 @@ UNIT = "positions/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel, from the ncu captures
-# summarised under profiles/ (None where no capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"single_request": 1.0406e9, "batched_serving": 2.193e9}
+# summarised under profiles/, keyed by (workload, kernel): a capture of another kernel does not count.
+NCU_TRAFFIC = {
+    ("single_request", "confidence_tc_kernel"): (1.0406e9, "profiles/confidence_tc_single_request.md"),
+    ("batched_serving", "confidence_tc_kernel"): (2.193e9, "profiles/confidence_tc_batched_serving.md"),
+}
 
 
 def load_peaks():
@@ -126,6 +135,28 @@ def ridge_rows(peaks) -> float:
     return peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
 
 
+# ------------------------------------------------------------------------------------ shared by both arms
+
+def config_dict(cfg, n_gpus):
+    """The `config` object of the JSON line: the same keys and values in the library arm and in the
+    reference arm, so that the two lines can be matched."""
+    return {"workload": cfg.name, "B": cfg.B, "D": cfg.D, "M": cfg.M, "H": cfg.H, "V": cfg.V, "rows": cfg.rows,
+            "policy": {"tau": cfg.tau, "k_min": cfg.k_min, "k_max": cfg.k_max, "stride": cfg.stride},
+            "parallelism": f"replicas x{n_gpus}",
+            "l2": f"inputs larger than L2: W is {cfg.V * cfg.H * 2 / 1e6:.0f} MB and is re-read every step"}
+
+
+def resolve_config(name, blocks=0):
+    import psd_inputs as gen
+    if name.startswith("deep_sweep_D"):
+        cfg = gen.with_depth(gen.CONFIGS["deep_sweep"], int(name.rsplit("D", 1)[1]))
+    else:
+        cfg = gen.CONFIGS[name]
+    if blocks > 0:
+        cfg = replace(cfg, B=blocks, name=f"{cfg.name}_B{blocks}")
+    return cfg
+
+
 # ------------------------------------------------------------------------------------ reference arm
 
 def oracle_sample_rate(cfg, wl, n_rows):
@@ -177,16 +208,13 @@ def cpu_baseline(cfg, wl, budget_s=15.0):
                       f"all {cfg.V} vocabulary entries), {secs:.2f} s"}
 
 
-def run_reference(args, cfg):
-    """--impl reference: the CPU oracle, K timed steps, each a bounded sample of the workload."""
+def reference_workload(args, cfg, total_budget):
+    """The CPU oracle on one workload: K timed steps after W warm-ups, each step a bounded sample of
+    the workload sized so that all of them fit `total_budget` seconds.  Returns the result object."""
     import oracle
     import psd_inputs as gen
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return 0
     wl = gen.make(cfg)
     t_probe = oracle_sample_rate(cfg, wl, 1)
-    total_budget = 150.0
     rows_per_step = int(max(1, min(cfg.rows, total_budget / max(t_probe, 1e-9) / (args.steps + args.warmup))))
     rows_per_block = cfg.D * cfg.M
     po = oracle_policy(cfg)
@@ -208,39 +236,47 @@ def run_reference(args, cfg):
         secs += s
         rows += r
     value = rows / secs
-    sample = (f"each step = the whole oracle step on {n_blocks} block(s)" if whole_blocks else
+    sample = (f"each step = the whole oracle step on {n_blocks} of {cfg.B} block(s)" if whole_blocks else
               f"each step = the oracle's confidence computation on {rows_per_step} row(s) "
               f"(fewer than one block of {rows_per_block}; the integer stages need whole blocks)")
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "D": cfg.D, "M": cfg.M, "H": cfg.H, "V": cfg.V,
-                       "rows_per_step": int(rows / args.steps)},
+    sample += f"; {int(rows / args.steps)} of {cfg.rows} rows per step"
+    return {"value": value, "unit": UNIT, "ms_per_step": 1e3 * secs / args.steps,
+            "config": config_dict(cfg, args.gpus),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
                              "sample": sample},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def run_reference(args, names):
+    """--impl reference: the CPU oracle on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    budgets = [150.0] if len(names) == 1 else [100.0] + [50.0] * (len(names) - 1)
+    results = [reference_workload(args, resolve_config(n, args.blocks), b) for n, b in zip(names, budgets)]
+    top = results[0]
+    line = {"impl": "reference", "metric": METRIC, "value": top["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": top["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": top["config"], "cpu_baseline": top["cpu_baseline"], "e2e": top["e2e"],
             "gpu_launches": 0}
+    for r in results[1:]:
+        line[r["config"]["workload"]] = r
     print(json.dumps(line), flush=True)
     return 0
 
 
 # ------------------------------------------------------------------------------------ our arm
 
-def run_ours(args, cfg):
+BAD_REASONS = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+
+
+def measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseline):
+    """All measurements of one workload on this rank's GPU; rank 0 gets the result object back."""
     import torch
 
     import paper_2605_15609_b200 as psd
     import psd_inputs as gen
     from paper_2605_15609_b200 import replicas
-
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
-    info = replicas.rank_info_from_env()
-    torch.cuda.set_device(info.local_rank)
-    device = torch.device("cuda", info.local_rank)
-    replicas.init_process_group(info)
-    peaks, peaks_kind = load_peaks()
 
     # Every replica holds the same W; each rank has its own batch of blocks.
     W = gen.weights(cfg)
@@ -274,6 +310,8 @@ def run_ours(args, cfg):
     first = {k: getattr(buf, k).clone() for k in ("sigma", "n_fill", "draft_tokens", "draft_mask")}
 
     def timed_region(step_fn, n):
+        """Exactly n steps between two events on the launching stream, barrier + synchronize on both
+        sides; returns this region's duration as the max over ranks."""
         replicas.barrier(info, device)
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -283,7 +321,20 @@ def run_ours(args, cfg):
         e1.record(stream)
         torch.cuda.synchronize()
         replicas.barrier(info, device)
-        return e0.elapsed_time(e1) * 1e-3
+        return replicas.max_over_ranks(e0.elapsed_time(e1) * 1e-3, info, device)
+
+    def repeated(step_fn, n):
+        """The n-step region repeated until args.min_seconds of device time have passed (at least 3
+        times); all ranks run the same number of repeats because they share the max-over-ranks times."""
+        times = []
+        while len(times) < 3 or (sum(times) < args.min_seconds and len(times) < 5000):
+            times.append(timed_region(step_fn, n))
+        return times
+
+    def spread(times, n):
+        return {"ms_per_step_median": 1e3 * statistics.median(times) / n, "ms_per_step_min": 1e3 * min(times) / n,
+                "ms_per_step_max": 1e3 * max(times) / n, "repeats": len(times), "steps_per_repeat": n,
+                "timed_seconds": sum(times)}
 
     # ---- device-resident steps: the headline value
     for _ in range(args.warmup):
@@ -293,29 +344,31 @@ def run_ours(args, cfg):
         sampler = ClockSampler(physical_gpu_index(info.local_rank))
         launches0 = psd.psd_launch_count()
         sampler.start()
-        secs = timed_region(lambda i: psd.psd_step(buf, pg, ws, status, stream), args.steps)
+        times = repeated(lambda i: psd.psd_step(buf, pg, ws, status, stream), args.steps)
         sampler.sample()
         sampler.stop()
         launches = psd.psd_launch_count() - launches0
-        # a timed region that saw a hardware or thermal slowdown is taken again, once
-        bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(sampler.summary()["reasons"])
+        # a measurement that saw a hardware or thermal slowdown is taken again, once
+        bad = BAD_REASONS & set(sampler.summary()["reasons"])
         bad_anywhere = replicas.max_over_ranks(1.0 if bad else 0.0, info, device) > 0   # all ranks decide alike
         if not bad_anywhere or remeasured:
             break
         remeasured = True
         time.sleep(2.0)
     if int(status.item()) != 0:
-        raise RuntimeError("device status: " + psd.status_string(int(status.item())))
-    value, secs_max = replicas.aggregate_throughput(float(R) * args.steps, secs, info, device)
+        code = int(status.item())
+        raise RuntimeError("device status: " + (psd.status_string(code) if code < 0 else f"{code} non-finite rows"))
+    secs_region = statistics.median(times)
+    rows_all = replicas.sum_over_ranks(float(R) * args.steps, info, device)
+    value = rows_all / secs_region
+    timed_total = sum(times)
 
     if args.profile_only:
-        if info.is_main:
-            print(json.dumps({"profile_only": True, "workload": cfg.name, "ms_per_step": 1e3 * secs_max / args.steps,
-                              "gpu_launches": launches}), flush=True)
-        return 0
+        return {"profile_only": True, "workload": cfg.name, "ms_per_step": 1e3 * secs_region / args.steps,
+                "gpu_launches": launches}
 
-    # ---- the same region again with an event pair around the fused kernel of every step
-    n_k = min(args.steps, 512)
+    # ---- the same steps again with an event pair around the fused kernel of every step
+    n_k = max(8, min(args.steps * len(times), 512))
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
     for a, b in evs:          # torch creates the CUDA event on first record; the library re-records it later
         a.record(stream)
@@ -335,11 +388,10 @@ def run_ours(args, cfg):
     for k, v in first.items():
         getattr(hb, k).copy_(v)
     staging = torch.empty(psd.psd_step_host_bytes(B, M, H, V, D), dtype=torch.uint8, device=device)
-    n_e2e = max(3, min(args.steps, 200))
     for _ in range(3):
         psd.psd_step_host(hb, pg, staging, stream)
-    secs_e2e = timed_region(lambda i: psd.psd_step_host(hb, pg, staging, stream), n_e2e)
-    e2e_value, _ = replicas.aggregate_throughput(float(R) * n_e2e, secs_e2e, info, device)
+    times_e2e = repeated(lambda i: psd.psd_step_host(hb, pg, staging, stream), args.steps)
+    e2e_value = rows_all / statistics.median(times_e2e)
     # bytes actually moved per step: hidden plus the draft state up (one block, padding included), every
     # output and the status word down (one block)
     _, off = psd.psd_step_host_block(B, M, D)
@@ -347,41 +399,81 @@ def run_ours(args, cfg):
     d2h = off[14] + 4
 
     if not info.is_main:
-        return 0
+        return None
 
     tensor_bound = R > ridge_rows(peaks)
+    kernel_name = psd.psd_confidence_kernel_name(R)
     if tensor_bound:
-        peak = peaks["bf16_tflops_sustained"] if secs_max > 1.0 else peaks["bf16_tflops"]
+        # back-to-back tensor-bound steps for over a second sit at the board's power cap: the sustained
+        # cuBLAS figure is the like-for-like peak there, the burst figure otherwise; both fractions are given
+        sustained = timed_total > 1.0
+        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
         achieved = algorithmic_flops(cfg) / kernel_s / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_kind": f"{'sustained' if secs_max > 1.0 else 'burst'} bf16, of {peaks_kind}",
-                "frac_of_burst": achieved / peaks["bf16_tflops"]}
+                "peak_kind": f"{'sustained' if sustained else 'burst'} bf16, of {peaks_kind}",
+                "frac_of_burst": achieved / peaks["bf16_tflops"],
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"]}
     else:
         peak = peaks["hbm_gbs"]
         achieved = algorithmic_bytes(cfg) / kernel_s / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"copy bandwidth, of {peaks_kind}"}
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(cfg.name)
-    roof["kernel"] = "confidence_tc_kernel"
+    traffic = NCU_TRAFFIC.get((cfg.name, kernel_name))
+    roof["traffic"] = traffic[0] if traffic else None
+    roof["traffic_source"] = (f"ncu capture summarised in {traffic[1]}; not measured by this run" if traffic else
+                              "no ncu capture of this kernel on this workload")
+    roof["kernel"] = kernel_name
     roof["kernel_ms"] = kernel_s * 1e3
+    roof["kernel_ms_min"] = min(kernel_ms)
+    roof["kernel_ms_max"] = max(kernel_ms)
     roof["kernel_launches_timed"] = n_k
     roof["step_ms_while_instrumented"] = 1e3 * secs_instr / n_k
     roof["algorithmic_bytes"] = algorithmic_bytes(cfg)
     roof["algorithmic_flops"] = algorithmic_flops(cfg)
 
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": info.world_size, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * secs_max / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": B, "D": D, "M": M, "H": H, "V": V, "rows": R,
-                       "policy": {"tau": cfg.tau, "k_min": cfg.k_min, "k_max": cfg.k_max, "stride": cfg.stride},
-                       "parallelism": f"replicas x{info.world_size}",
-                       "l2": f"inputs larger than L2: W is {V * H * 2 / 1e6:.0f} MB and is re-read every step"},
-            "clocks": dict(sampler.summary(), remeasured=remeasured),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": 1e3 * secs_e2e / n_e2e, "steps": n_e2e},
-            "gpu_launches": launches,
-            "roofline": roof,
-            "cpu_baseline": cpu_baseline(cfg, wl)}
+    res = {"value": value, "unit": UNIT, "ms_per_step": 1e3 * secs_region / args.steps,
+           "timing": spread(times, args.steps), "config": config_dict(cfg, info.world_size),
+           "clocks": dict(sampler.summary(), remeasured=remeasured),
+           "e2e": dict({"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "ms_per_step": 1e3 * statistics.median(times_e2e) / args.steps, "steps": args.steps},
+                       **{"timing": spread(times_e2e, args.steps)}),
+           "gpu_launches": launches // len(times), "gpu_launches_all_repeats": launches, "roofline": roof}
+    if with_cpu_baseline:
+        res["cpu_baseline"] = cpu_baseline(cfg, wl)
+    return res
+
+
+def run_ours(args, names):
+    import torch
+
+    from paper_2605_15609_b200 import replicas
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    info = replicas.rank_info_from_env()
+    torch.cuda.set_device(info.local_rank)
+    device = torch.device("cuda", info.local_rank)
+    replicas.init_process_group(info)
+    peaks, peaks_kind = load_peaks()
+
+    results = []
+    for i, name in enumerate(names):
+        cfg = resolve_config(name, args.blocks)
+        results.append(measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseline=(i == 0)))
+        torch.cuda.empty_cache()
+    if not info.is_main:
+        return 0
+    top = results[0]
+    if args.profile_only:
+        print(json.dumps(top), flush=True)
+        return 0
+    line = {"metric": METRIC, "value": top["value"], "unit": UNIT, "n_gpus": info.world_size, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": top["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
+    line.update({k: top[k] for k in ("config", "timing", "clocks", "e2e", "gpu_launches", "gpu_launches_all_repeats",
+                                     "roofline", "cpu_baseline")})
+    for r in results[1:]:
+        line[r["config"]["workload"]] = r
     print(json.dumps(line), flush=True)
     return 0
 
@@ -452,16 +544,24 @@ def run_loop(args, cfg):
     return 0
 
 
+DEFAULT_WORKLOADS = ("batched_serving", "single_request")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", default="single_request",
-                    help="workload: tiny, single_request, class_7b, batched_serving, deep_sweep[_D1|_D2|_D4]")
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default=None,
+                    help="one workload: tiny, single_request, class_7b, batched_serving, deep_sweep[_D1|_D2|_D4]. "
+                         "Default: batched_serving (8192 rows, tensor bound) as the line's own result, with "
+                         "single_request (128 rows, HBM bound) measured the same way under the key of that name")
     ap.add_argument("--blocks", type=int, default=0,
                     help="override the workload's number of blocks B (rows = B*D*M), e.g. to sweep row counts "
                          "across the HBM/tensor ridge; the printed config names the override")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="the K-step timed region is repeated until this much device time has passed (at least "
+                         "3 times); the line reports the median region and the spread")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loop", default=None, choices=["one_pass", "two_passes"],
                     help="time the whole decoding loop (psd_decode_blocks) instead of one step; an extra "
@@ -474,19 +574,14 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    import psd_inputs as gen
-    name = args.config
-    if name.startswith("deep_sweep_D"):
-        cfg = gen.with_depth(gen.CONFIGS["deep_sweep"], int(name.rsplit("D", 1)[1]))
-    else:
-        cfg = gen.CONFIGS[name]
-    if args.blocks > 0:
-        cfg = replace(cfg, B=args.blocks, name=f"{cfg.name}_B{args.blocks}")
+    if args.profile_only:
+        args.min_seconds = 0.0
+    names = [args.config] if args.config else list(DEFAULT_WORKLOADS)
     if args.impl == "reference":
-        return run_reference(args, cfg)
+        return run_reference(args, names)
     if args.loop:
-        return run_loop(args, cfg)
-    return run_ours(args, cfg)
+        return run_loop(args, resolve_config(names[-1], args.blocks))
+    return run_ours(args, names)
 
 
 if __name__ == "__main__":

@@ -12,7 +12,13 @@
  *
  * Conventions, common to every entry point unless it says otherwise:
  *   - Every array pointer is a DEVICE pointer owned by the caller.  The library allocates no
- *     device memory and keeps no state between calls.
+ *     device memory.  The computing entry points keep no state between calls; the only state the
+ *     library holds is a handful of process-wide settings (psd_set_confidence_impl, psd_set_tuning)
+ *     and a per-thread profiling hook (psd_set_kernel_events), all listed at the end of this file.
+ *     The settings are plain atomics read at the start of a call: changing one while another thread
+ *     is inside a call is not supported (PSD_TUNE_COMPACT_ROWS, for one, changes how much workspace
+ *     psd_step needs and which entries of tokV / confV it writes), so set them before the threads
+ *     that compute are started, or serialise.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
  *     default stream).  Outputs are valid once the stream has reached the end of the call.
  *   - The return value is PSD_OK or a negative psd_status code.  Argument errors are detected
@@ -47,6 +53,17 @@ typedef enum psd_status {
     PSD_ERR_TIMEOUT = -8      /* device side only, via status_dev: a bounded wait inside a kernel
                                  ran out; the kernel returned early and its outputs are invalid    */
 } psd_status;
+
+/*
+ * The device status word (`status_dev` of the entry points that take one): a device int32 that the
+ * CALLER zeroes.  After the call it holds
+ *     < 0   a psd_status code detected on the device (PSD_ERR_TIMEOUT); it is never overwritten;
+ *     > 0   PSD_ERR_NONFINITE count: the number of scored rows whose logits held a NaN or an infinity,
+ *           so that their confidence is NaN (such a row ranks below every number in the policy and
+ *           never exceeds tau; nothing faults);
+ *       0   neither.
+ * Counts of successive calls add up when the word is not zeroed in between.
+ */
 
 /* Limits checked by the entry points. */
 #define PSD_MAX_M 1024     /* slots per block                        */
@@ -112,9 +129,9 @@ size_t psd_compact_workspace_bytes(int32_t n_rows, int32_t H, int32_t V);
  *   out_token    [n_rows] int32;  out_conf [n_rows] fp32;  out_lse [n_rows] fp32 or NULL
  *   workspace    >= psd_workspace_bytes(n_rows, H, V) bytes, 256-byte aligned, device; contents
  *                are overwritten; concurrent calls need distinct workspaces
- *   status_dev   NULL, or a device int32 that the caller zeroed: receives PSD_ERR_TIMEOUT if a
- *                bounded wait inside the kernel expired (outputs are then invalid)
- * Rows whose logits contain NaN produce out_conf = NaN.
+ *   status_dev   NULL, or the device status word (see above): PSD_ERR_TIMEOUT if a bounded wait inside
+ *                the kernel expired (outputs are then invalid), else the number of non-finite rows
+ * Rows whose logits contain NaN produce out_conf = NaN and are counted in status_dev.
  */
 int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_ids,
                    int32_t n_rows, int32_t H, int32_t V,
@@ -150,7 +167,8 @@ int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const 
  * psd_merge_partials: max, sumexp, arg are [n_shards, n_rows] (shard-major, e.g. the all-gathered
  *   outputs of psd_confidence_partial); out_token, out_conf, out_lse as for psd_confidence.  Equal
  *   maxima keep the lowest global index, so the result does not depend on the number of shards
- *   beyond the rounding order of the sums.
+ *   beyond the rounding order of the sums.  All its arrays are 4-byte aligned (PSD_ERR_ALIGN otherwise);
+ *   it takes no status word (psd_confidence_partial has counted the non-finite rows of its shard).
  */
 int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, int32_t n_rows, int32_t H,
                            int32_t V_shard, int32_t v_offset, float* out_max, float* out_sumexp, int32_t* out_arg,
@@ -237,8 +255,11 @@ int psd_verify_accept(const int32_t* tokV, const float* confV,
  *     rejected with PSD_ERR_WORKSPACE (e.g. 128 rows x V = 126464 needs 1.5 MB and fits;
  *     8192 rows do not);
  *   - the first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress, with that device current); make that first call outside of any
- *     stream capture;
+ *     (cudaGetSymbolAddress, with that device current).  CUDA loads a library's device code lazily
+ *     by default, so this look-up can be the moment the driver loads the module and reserves the
+ *     array's memory: make one call per device at start-up, BEFORE the process hands the rest of
+ *     the device memory to its pool and outside of any stream capture.  A first call made after
+ *     the memory is gone fails with PSD_ERR_CUDA.  Later calls on that device touch no allocator;
  *   - it calls no cudaMalloc, cudaFree or other allocating routine;
  *   - all calls on a device share the one array, which keeps the previous call's contents.
  *     Nothing in it needs clearing (every entry read is written first by the same call), but two
@@ -493,6 +514,13 @@ int psd_set_tuning(int knob, int value);
  * clears itself.  Passing NULLs clears it.  Always returns PSD_OK.
  */
 int psd_set_kernel_events(void* start_event, void* stop_event);
+
+/*
+ * Name of the kernel that psd_confidence (and psd_step) launches for a batch of n_rows rows under the
+ * current psd_set_confidence_impl setting: "confidence_tc_kernel", "confidence_tc2_kernel" or
+ * "confidence_simt_kernel" (static storage).  For reports: it computes nothing.
+ */
+const char* psd_confidence_kernel_name(int32_t n_rows);
 
 /* Number of kernel launches the library has issued in this process (all entry points). */
 int64_t psd_launch_count(void);

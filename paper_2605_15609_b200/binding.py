@@ -8,7 +8,6 @@ raises.
 from __future__ import annotations
 
 import ctypes
-import os
 from dataclasses import dataclass
 
 import torch
@@ -65,10 +64,9 @@ class PsdError(RuntimeError):
 
 
 def _load() -> ctypes.CDLL:
-    path = _build.LIB
-    if not os.path.exists(path):
-        path = _build.build()
-    lib = ctypes.CDLL(path)
+    # build() compares the library's time stamp with the sources' and recompiles when a source is newer,
+    # so a stale library is never loaded silently
+    lib = ctypes.CDLL(_build.build())
     pol = PsdPolicy
     lib.psd_status_string.restype = ctypes.c_char_p
     lib.psd_status_string.argtypes = [ctypes.c_int]
@@ -128,6 +126,8 @@ def _load() -> ctypes.CDLL:
     lib.psd_set_tuning.argtypes = [ctypes.c_int, ctypes.c_int]
     lib.psd_set_kernel_events.restype = ctypes.c_int
     lib.psd_set_kernel_events.argtypes = [_vp, _vp]
+    lib.psd_confidence_kernel_name.restype = ctypes.c_char_p
+    lib.psd_confidence_kernel_name.argtypes = [_i32]
     lib.psd_launch_count.restype = _i64
     lib.psd_launch_count.argtypes = []
     return lib
@@ -194,6 +194,11 @@ def psd_set_kernel_events(start_event, stop_event) -> int:
             return None
         return e.cuda_event if hasattr(e, "cuda_event") else int(e)
     return int(LIB.psd_set_kernel_events(h(start_event), h(stop_event)))
+
+
+def psd_confidence_kernel_name(n_rows: int) -> str:
+    """Name of the kernel the confidence pass launches for ``n_rows`` rows under the current setting."""
+    return LIB.psd_confidence_kernel_name(int(n_rows)).decode()
 
 
 def psd_launch_count() -> int:

@@ -23,6 +23,16 @@ __device__ __forceinline__ void merge_triple(Triple& x, float m, float s, int32_
     }
 }
 
+// status word: a negative value is an error code and stays; otherwise it counts non-finite rows
+__device__ __forceinline__ void count_nonfinite_row(int32_t* status_dev) {
+    int32_t v = *reinterpret_cast<volatile int32_t*>(status_dev);
+    while (v >= 0 && v < INT32_MAX) {
+        const int32_t seen = atomicCAS(status_dev, v, v + 1);
+        if (seen == v) break;
+        v = seen;
+    }
+}
+
 constexpr int kCombineRows = 32;   // rows handled by one group of threads
 constexpr int kCombineLanes = 8;   // threads per row
 constexpr int kCombineThreads = kCombineRows * kCombineLanes;
@@ -37,7 +47,8 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
                                                int row0, int row_end, int g, Triple (*sh)[kCombineRows],
                                                int32_t* __restrict__ out_token, float* __restrict__ out_conf,
                                                float* __restrict__ out_lse, const int32_t* __restrict__ pos = nullptr,
-                                               float* __restrict__ out_max = nullptr, int32_t arg_offset = 0) {
+                                               float* __restrict__ out_max = nullptr, int32_t arg_offset = 0,
+                                               int32_t* status_dev = nullptr) {
     const int tx = g & 31, lane = g >> 5;
     const int out_row = row0 + tx;
     // with compacted rows the partials of output row r sit in column pos[r]; -1 = the row was not scored
@@ -83,6 +94,8 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
             out_conf[out_row] = 1.0f / x.s;
             if (out_lse) out_lse[out_row] = x.m + logf(x.s);
         }
+        // A row whose logits held a NaN or an infinity has no defined confidence: count it.
+        if (status_dev && !(isfinite(x.m) && isfinite(x.s))) count_nonfinite_row(status_dev);
     }
     __syncthreads();
 }

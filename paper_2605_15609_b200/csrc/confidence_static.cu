@@ -4,8 +4,10 @@
 // serving process that handed all free HBM to its own pool at start-up, or a plug-in called back
 // from inside another runtime where cudaMalloc (and the device-wide synchronisation it implies) is
 // off limits.  For them the per-split partial triples live in a fixed array that is part of the
-// library image: every GPU that loads the library carries PSD_STATIC_SCRATCH_BYTES of it until the
-// process exits, whether or not this entry point is ever called.
+// library image: every GPU that loads this part of the library carries PSD_STATIC_SCRATCH_BYTES of
+// it until the process exits.  With CUDA's default lazy loading the driver reserves the array when
+// the module is first needed on a device, which can be as late as the first call here: such callers
+// make one call per device at start-up, before they give the remaining memory away.
 #include <mutex>
 #include "psd_internal.cuh"
 
@@ -55,5 +57,5 @@ extern "C" int psd_confidence_static(const void* hidden_bf16, const void* w_lm_b
     psd::Partials part = psd::carve_partials(scratch, n_rows, V);
     const int n_split = psd::launch_confidence_tc(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st);
     if (n_split < 0) return n_split;
-    return psd::launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st);
+    return psd::launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, nullptr, nullptr, 0, status_dev);
 }

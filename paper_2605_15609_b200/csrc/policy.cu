@@ -254,6 +254,7 @@ struct StepTailArgs {
     float* confV;
     int32_t *sigma, *n_fill, *draft_tokens, *draft_mask;
     int32_t *tokens, *mask, *k_star, *n_spec, *n_comm, *sel, *n_sel, *sel_pos;
+    int32_t* status_dev;   // NULL, or the status word that counts non-finite rows
 };
 
 __global__ void step_tail_kernel(const StepTailArgs a) {
@@ -280,7 +281,7 @@ __global__ void step_tail_kernel(const StepTailArgs a) {
         const int r0 = c < n_chunks ? row_begin + c * kCombineRows : row_end;
         if (grp < groups)
             combine_rows32(a.pm, a.ps, a.pa, a.n_split, a.n_rows, r0, row_end, g, sh[grp], a.tokV, a.confV,
-                           nullptr, a.pos);
+                           nullptr, a.pos, nullptr, 0, a.status_dev);
     }
     __syncthreads();
 
@@ -334,9 +335,10 @@ int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_p
                      int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
                      int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
                      int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st,
-                     const int32_t* pos) {
+                     const int32_t* pos, int32_t* status_dev) {
     StepTailArgs a;
     a.pos = pos;
+    a.status_dev = status_dev;
     a.pm = part.m; a.ps = part.s; a.pa = part.a;
     a.n_split = n_split; a.n_rows = n_rows; a.M = M; a.p = p;
     a.tokV = tokV; a.confV = confV;

@@ -31,6 +31,11 @@ bool conf_shape_ok(int n_rows, int H, int V) {
 }
 }  // namespace
 
+// Default choice by measurement (V = 126464, H = 4096): see launch_confidence_tc.
+static bool confidence_uses_pairs(int impl, int n_rows) {
+    return impl == 3 || (impl == 0 && n_rows > 128 && n_rows <= 256);
+}
+
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 int pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 long long band_bytes() { return g_band_bytes.load(std::memory_order_relaxed); }
@@ -42,7 +47,7 @@ int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, i
     // Default choice by measurement (V = 126464, H = 4096): at 129..256 rows one CTA pair covers both row
     // tiles and fetches every W tile once (258-265 us against 276-282 us); at 128 rows and below, and
     // from 257 rows up, the single-CTA kernel is faster or equal (see confidence_tc2.cu).
-    const bool pairs = impl == 3 || (impl == 0 && n_rows > 128 && n_rows <= 256);
+    const bool pairs = confidence_uses_pairs(impl, n_rows);
     return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st)
                  : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st);
 }
@@ -116,6 +121,12 @@ int psd_set_kernel_events(void* start_event, void* stop_event) {
     return PSD_OK;
 }
 
+const char* psd_confidence_kernel_name(int32_t n_rows) {
+    const int impl = g_conf_impl.load(std::memory_order_relaxed);
+    if (impl == 1) return "confidence_simt_kernel";
+    return confidence_uses_pairs(impl, n_rows) ? "confidence_tc2_kernel" : "confidence_tc_kernel";
+}
+
 int64_t psd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_ids,
@@ -149,7 +160,7 @@ int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t
         if (e != cudaSuccess) return PSD_ERR_CUDA;
     }
     if (n_split < 0) return n_split;
-    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st);
+    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, nullptr, nullptr, 0, status_dev);
 }
 
 int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_mask,
@@ -180,7 +191,7 @@ int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const 
         if (e != cudaSuccess) return PSD_ERR_CUDA;
     }
     if (n_split < 0) return n_split;
-    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, cs.pos);
+    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, cs.pos, nullptr, 0, status_dev);
 }
 
 int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, int32_t n_rows, int32_t H,
@@ -199,13 +210,16 @@ int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, in
                       ? launch_confidence_simt(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, st)
                       : launch_confidence_tc(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, status_dev, st);
     if (n_split < 0) return n_split;
-    return launch_combine(part, n_split, n_rows, out_arg, out_sumexp, nullptr, st, nullptr, out_max, v_offset);
+    return launch_combine(part, n_split, n_rows, out_arg, out_sumexp, nullptr, st, nullptr, out_max, v_offset, status_dev);
 }
 
 int psd_merge_partials(const float* max, const float* sumexp, const int32_t* arg, int32_t n_shards, int32_t n_rows,
                        int32_t* out_token, float* out_conf, float* out_lse, void* cuda_stream) {
     if (!max || !sumexp || !arg || !out_token || !out_conf) return PSD_ERR_NULL;
     if (n_shards < 1 || n_rows < 1) return PSD_ERR_SHAPE;
+    if (!aligned(max, 4) || !aligned(sumexp, 4) || !aligned(arg, 4) || !aligned(out_token, 4) ||
+        !aligned(out_conf, 4) || !aligned(out_lse, 4))
+        return PSD_ERR_ALIGN;
     Partials part;
     part.m = const_cast<float*>(max);
     part.s = const_cast<float*>(sumexp);
@@ -310,10 +324,10 @@ static int step_impl(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, i
     if (!g)
         return launch_step_tail(part, n_split, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
                                 io->draft_tokens, io->draft_mask, io->tokens, io->mask, io->k_star,
-                                io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st, pos);
+                                io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st, pos, status_dev);
     // draft graph: the same stages as separate launches (merge, acceptance over the graph, policy on
     // node k*, next drafts of the graph)
-    if (int e = launch_combine(part, n_split, n_rows, io->tokV, io->confV, nullptr, st, pos)) return e;
+    if (int e = launch_combine(part, n_split, n_rows, io->tokV, io->confV, nullptr, st, pos, nullptr, 0, status_dev)) return e;
     if (int e = psd_verify_accept_dag(io->tokV, io->confV, io->sigma, io->draft_tokens, io->draft_mask, B, M, p, g,
                                       io->tokens, io->mask, io->k_star, io->n_spec_accepted, io->n_committed,
                                       nullptr, cuda_stream))

@@ -88,9 +88,10 @@ inline CompactSpace carve_compact(void* workspace, int n_rows, int H, int V) {
 // and its outputs are left alone).
 int launch_combine(Partials part, int n_split, int n_rows,
                    int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st,
-                   const int32_t* pos = nullptr, float* out_max = nullptr, int32_t arg_offset = 0);
+                   const int32_t* pos = nullptr, float* out_max = nullptr, int32_t arg_offset = 0,
+                   int32_t* status_dev = nullptr);
 // With out_max the kernel writes the merged triple instead: out_max = max, out_conf = sum-exp,
-// out_token = argmax + arg_offset.
+// out_token = argmax + arg_offset.  status_dev: NULL, or the status word that counts non-finite rows.
 
 // policy.cu
 int launch_select(const float* conf, const int32_t* tok, const int32_t* node, int n_nodes,
@@ -110,6 +111,6 @@ int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_p
                      int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
                      int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
                      int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st,
-                     const int32_t* pos = nullptr);
+                     const int32_t* pos = nullptr, int32_t* status_dev = nullptr);
 
 }  // namespace psd

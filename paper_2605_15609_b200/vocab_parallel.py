@@ -25,6 +25,19 @@ def shard_rows(V: int, world_size: int, rank: int, multiple: int = 16):
     return min(u0 * multiple, V), min(u1 * multiple, V)
 
 
+EMPTY_ARG = 2**31 - 1   # argmax of a rank that holds no vocabulary rows: loses every tie
+
+
+def neutral_triple(n_rows: int, device="cpu") -> torch.Tensor:
+    """Packed triples ``[3, n_rows]`` of an empty vocabulary range: max = -inf, sum-exp = 0, argmax =
+    EMPTY_ARG.  Merging it into any other triple leaves that triple unchanged."""
+    t = torch.empty(3, n_rows, dtype=torch.int32, device=device)
+    t[0].view(torch.float32).fill_(float("-inf"))
+    t[1].zero_()
+    t[2].fill_(EMPTY_ARG)
+    return t
+
+
 def gather_partials(local: torch.Tensor, group=None) -> torch.Tensor:
     """All-gathers one rank's packed triples ``[3, n_rows]`` (int32 words: the bit patterns of max and
     sum-exp, then the argmax) into ``[world, 3, n_rows]``, rank-major."""
@@ -46,18 +59,33 @@ class VocabParallelHead:
         dev = w_shard.device
         H = w_shard.shape[1]
         self.local = torch.zeros(3, max_rows, dtype=torch.int32, device=dev)
-        self.ws = torch.empty(psd.psd_workspace_bytes(max_rows, H, w_shard.shape[0]), dtype=torch.uint8, device=dev)
+        self.ws = torch.empty(max(256, psd.psd_workspace_bytes(max_rows, H, max(1, w_shard.shape[0]))),
+                              dtype=torch.uint8, device=dev)
+        self._m = self._s = self._a = None
         self.max_rows = max_rows
 
     def confidence(self, hidden, out_token, out_conf, out_lse=None, status=None, stream=None):
+        """Whole-vocabulary prediction and confidence of every row of ``hidden`` on every rank.  All
+        three steps (this rank's partial pass, the all-gather, the merge) are ordered on ``stream``
+        (default: torch's current stream): the collective and the temporaries are issued with that
+        stream current, and the gathered triples are kept as members until the next call so that the
+        allocator cannot hand their memory out while the merge still reads it."""
         n = hidden.shape[0]
         if n > self.max_rows:
             raise ValueError("more rows than the head was sized for")
-        loc = self.local[:, :n] if n == self.max_rows else self.local.view(-1)[:3 * n].view(3, n)
-        self.psd.psd_confidence_partial(hidden, self.w, self.v_offset, loc[0].view(torch.float32),
-                                        loc[1].view(torch.float32), loc[2], self.ws, status, stream)
-        allp = gather_partials(loc, self.group)                  # [world, 3, n]
-        m = allp[:, 0].contiguous().view(torch.float32)
-        s = allp[:, 1].contiguous().view(torch.float32)
-        a = allp[:, 2].contiguous()
-        self.psd.psd_merge_partials(m, s, a, out_token, out_conf, out_lse, stream)
+        stream = torch.cuda.current_stream(self.w.device) if stream is None else stream
+        with torch.cuda.stream(stream):
+            loc = self.local[:, :n] if n == self.max_rows else self.local.view(-1)[:3 * n].view(3, n)
+            if self.w.shape[0] == 0:
+                # an empty range of the vocabulary (more ranks than V / 16): the neutral triple
+                loc[0].view(torch.float32).fill_(float("-inf"))
+                loc[1].zero_()
+                loc[2].fill_(EMPTY_ARG)
+            else:
+                self.psd.psd_confidence_partial(hidden, self.w, self.v_offset, loc[0].view(torch.float32),
+                                                loc[1].view(torch.float32), loc[2], self.ws, status, stream)
+            allp = gather_partials(loc, self.group)                  # [world, 3, n]
+            self._m = allp[:, 0].contiguous().view(torch.float32)
+            self._s = allp[:, 1].contiguous().view(torch.float32)
+            self._a = allp[:, 2].contiguous()
+            self.psd.psd_merge_partials(self._m, self._s, self._a, out_token, out_conf, out_lse, stream)

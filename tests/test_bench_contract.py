@@ -8,6 +8,7 @@ import sys
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+CONFIG_KEYS = {"workload", "B", "D", "M", "H", "V", "rows", "policy", "parallelism", "l2"}
 COMMON = ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
           "vs_baseline", "dtype", "data", "config", "e2e", "gpu_launches", "cpu_baseline")
 
@@ -30,6 +31,15 @@ def test_reference_arm_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1 and d["cpu_baseline"]["sample"]
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
     assert d["e2e"]["value"] == d["value"] == d["cpu_baseline"]["value"]
+    assert set(d["config"]) == CONFIG_KEYS and d["config"]["rows"] == 128
+
+
+def test_default_run_names_the_largest_workload_and_nests_the_small_one():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.DEFAULT_WORKLOADS == ("batched_serving", "single_request")
+    big = bench.config_dict(bench.resolve_config("batched_serving"), 1)
+    assert big["rows"] == 8192 and set(big) == CONFIG_KEYS
 
 
 @pytest.mark.gpu
@@ -50,3 +60,8 @@ def test_library_arm_line():
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["value"] > 0 and c["cores"] >= 1 and c["sample"]
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    assert set(d["config"]) == CONFIG_KEYS                           # the same keys as the reference arm's
+    t = d["timing"]
+    assert t["repeats"] >= 3 and t["steps_per_repeat"] == 50 and t["timed_seconds"] >= 1.0
+    assert t["ms_per_step_min"] <= d["ms_per_step"] <= t["ms_per_step_max"]
+    assert r["kernel"] == "confidence_tc_kernel" and "traffic_source" in r

@@ -104,6 +104,31 @@ def test_nan_inputs_give_nan_confidence_not_a_fault():
     assert np.isnan(conf[3]) and np.isfinite(np.delete(conf, 3)).all()
 
 
+def test_non_finite_rows_are_counted_in_the_status_word():
+    hid, W = _rand_inputs(44, 300, 64, 2000)
+    hid = hid.copy()
+    hid[3, 5] = 0x7FC0                              # NaN
+    hid[140, 0] = 0x7F80                            # +inf: the logits of that row are +-inf
+    hid[299, 7] = 0xFFC0                            # -NaN
+    h, w = bf16_dev(hid), bf16_dev(W)
+    n, H = h.shape
+    for impl in (0, 1, 2, 3):
+        tok = torch.zeros(n, dtype=torch.int32, device="cuda")
+        conf = torch.zeros(n, dtype=torch.float32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ws = torch.empty(psd.psd_workspace_bytes(n, H, w.shape[0]), dtype=torch.uint8, device="cuda")
+        prev = psd.psd_set_confidence_impl(impl)
+        try:
+            psd.psd_confidence(h, w, tok, conf, None, ws, status)
+            psd.psd_confidence(h, w, tok, conf, None, ws, status)      # counts add up until the word is zeroed
+            torch.cuda.synchronize()
+        finally:
+            psd.psd_set_confidence_impl(prev)
+        c = conf.cpu().numpy()
+        assert int(status.item()) == 6
+        assert np.isnan(c[[3, 140, 299]]).all() and np.isfinite(np.delete(c, [3, 140, 299])).all()
+
+
 def _raw(hid, W):
     h, w = bf16_dev(hid), bf16_dev(W)
     n, H = h.shape

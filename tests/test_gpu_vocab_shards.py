@@ -90,3 +90,38 @@ def test_head_object_single_process():
     head.confidence(bf16_dev(hid), tok, conf, lse)
     torch.cuda.synchronize()
     check_confidence(np_(tok), np_(conf), np_(lse), tok_o, conf_o, lse_o, gap_o)
+
+
+def test_head_object_on_a_stream_that_is_not_current():
+    """The partial pass, the gather and the merge must all be ordered on the stream that is passed in, not
+    on torch's current stream: a long kernel is queued on the side stream first, so work that wrongly went
+    to the current stream would run ahead of the partial pass and read triples that are not written yet."""
+    R, H, V = 128, 256, 20000
+    hid, W = _inputs(11, R, H, V)
+    tok_o, conf_o, lse_o, gap_o = oracle.confidence(hid, W)
+    head = VocabParallelHead(bf16_dev(W), 0, max_rows=R)
+    h_dev = bf16_dev(hid)
+    tok = torch.full((R,), -3, dtype=torch.int32, device="cuda")
+    conf = torch.full((R,), -3.0, dtype=torch.float32, device="cuda")
+    lse = torch.full((R,), -3.0, dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    big = torch.empty(1 << 28, dtype=torch.float32, device="cuda")
+    with torch.cuda.stream(side):
+        for _ in range(4):
+            big.add_(1.0)                      # a few milliseconds of work ahead of the pass, on the side stream
+    head.confidence(h_dev, tok, conf, lse, stream=side)
+    side.synchronize()
+    check_confidence(np_(tok), np_(conf), np_(lse), tok_o, conf_o, lse_o, gap_o)
+
+
+def test_head_object_with_an_empty_range():
+    R, H = 16, 64
+    w = torch.zeros(0, H, dtype=torch.bfloat16, device="cuda")
+    head = VocabParallelHead(w, 640, max_rows=R)
+    tok = torch.zeros(R, dtype=torch.int32, device="cuda")
+    conf = torch.zeros(R, dtype=torch.float32, device="cuda")
+    # alone in its group the merged result is the neutral triple itself: the call must simply not fail
+    head.confidence(torch.zeros(R, H, dtype=torch.bfloat16, device="cuda"), tok, conf)
+    torch.cuda.synchronize()
+    assert (np_(tok) == 2**31 - 1).all()

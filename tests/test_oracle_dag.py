@@ -22,11 +22,14 @@ def _case(rng, B, M, K_sets, p_masked=0.8):
     return conf, tok, tokens, mask
 
 
+@pytest.mark.parametrize("accept_mode", [0, 1, 2])
 @pytest.mark.parametrize("D,step", [(1, 1), (4, 1), (3, 2), (5, 3)])
-def test_path_graph_with_immediate_edges_equals_the_chain(D, step):
+def test_path_graph_with_immediate_edges_equals_the_chain(D, step, accept_mode):
+    # the chain's three acceptance modes are pinned on their own (per-depth enumeration, the mode-2 hand
+    # case): on a path graph the graph's branch of every mode has to give the chain's result
     rng = np.random.default_rng(D * 10 + step)
     B, M = 6, 12
-    p = Policy(tau=0.5, k_min=step, k_max=0, depth=D, stride=step, mask_id=MASK)
+    p = Policy(tau=0.5, k_min=step, k_max=0, depth=D, stride=step, accept_mode=accept_mode, mask_id=MASK)
     conf, tok, tokens, mask = _case(rng, B, M, None)
     ranks = oracle.chain_as_dag(D, step)
     a = oracle.build_drafts(conf, tok, tokens, mask, p)
@@ -45,7 +48,19 @@ def test_path_graph_with_immediate_edges_equals_the_chain(D, step):
     assert (full[5] >= path[5]).all() and (full[3] >= path[3]).all()
 
 
-def _reachable_by_brute_force(tokV, confV, sigma_b, tok_t, node_ranks, tau, b):
+def _policy_slots_by_sorting(conf_q, masked_q, p):
+    """pi(parent's draft) restated with a numpy sort: among the slots still masked in the parent's draft,
+    ordered by (confidence descending, slot ascending), the first n, with n the number above tau clamped
+    to [k_min, k_max] and to the number of masked slots (Sec. 3.2 Stage 1; App. B.2)."""
+    slots = np.nonzero(masked_q)[0]
+    order = slots[np.lexsort((slots, -conf_q[slots]))]
+    n = max(int((conf_q[slots] > p.tau).sum()), p.k_min)
+    if p.k_max:
+        n = min(n, p.k_max)
+    return set(order[:min(n, len(order))].tolist())
+
+
+def _reachable_by_brute_force(tokV, confV, sigma_b, tok_t, node_ranks, p, b, draft_mask):
     """Accepted set from the definition: k is accepted iff there is a sequence root = q0, q1, .., k of
     nodes, each a strict superset of the one before, every step passing its checks."""
     K = len(node_ranks)
@@ -53,8 +68,17 @@ def _reachable_by_brute_force(tokV, confV, sigma_b, tok_t, node_ranks, tau, b):
     S = [frozenset(int(sigma_b[j]) for j in node_ranks[k] if j < m) for k in range(K)]
     nominal = [frozenset(s) for s in node_ranks]
 
+    def slot_ok(q, i):
+        if int(tokV[b, q, i]) != int(tok_t[i]):
+            return False
+        if p.accept_mode == 0:
+            return float(confV[b, q, i]) > p.tau
+        if p.accept_mode == 1:
+            return True
+        return i in _policy_slots_by_sorting(confV[b, q], draft_mask[b, q], p)
+
     def step_ok(q, k):
-        return all(int(tokV[b, q, i]) == int(tok_t[i]) and float(confV[b, q, i]) > tau for i in S[k] - S[q])
+        return all(slot_ok(q, i) for i in S[k] - S[q])
 
     acc = set()
     for k in range(K):
@@ -74,27 +98,29 @@ def _reachable_by_brute_force(tokV, confV, sigma_b, tok_t, node_ranks, tau, b):
     return acc, S
 
 
-def test_acceptance_equals_path_enumeration():
+@pytest.mark.parametrize("accept_mode,k_max", [(0, 0), (1, 0), (2, 0), (2, 2)])
+def test_acceptance_equals_path_enumeration(accept_mode, k_max):
     rng = np.random.default_rng(5)
     node_ranks = [set(), {0}, {1}, {0, 1}, {0, 2}, {0, 1, 2}]
     B, M = 40, 6
-    p = Policy(tau=0.5, k_min=1, depth=len(node_ranks), mask_id=MASK)
+    p = Policy(tau=0.5, k_min=1, k_max=k_max, depth=len(node_ranks), accept_mode=accept_mode, mask_id=MASK)
     conf, tok, tokens, mask = _case(rng, B, M, None, p_masked=0.9)
     sigma, n_fill, dt, dm = oracle.build_drafts_dag(conf, tok, tokens, mask, p, node_ranks)
     K = len(node_ranks)
     tokV = np.where(rng.random((B, K, M)) < 0.75, tok[:, None, :], 77).astype(np.int32)
-    confV = rng.random((B, K, M)) * 0.5 + 0.45
+    confV = rng.random((B, K, M)) * 0.5 + (0.45 if accept_mode == 0 else 0.25)
     tokens2, mask2, k_star, n_spec, n_comm, accepted = oracle.verify_accept_dag(tokV, confV, sigma, dt, dm, p,
                                                                                 node_ranks)
     seen_multi = 0
     for b in range(B):
-        acc, S = _reachable_by_brute_force(tokV, confV, sigma[b], tok[b], node_ranks, p.tau, b)
+        acc, S = _reachable_by_brute_force(tokV, confV, sigma[b], tok[b], node_ranks, p, b, dm)
         assert set(np.nonzero(accepted[b])[0].tolist()) == acc
         best = max(sorted(acc), key=lambda k: len(S[k]))
         assert len(S[k_star[b]]) == len(S[best]) == n_spec[b] and k_star[b] in acc
         assert k_star[b] == min(k for k in acc if len(S[k]) == n_spec[b])
         seen_multi += int(3 in acc and not (1 in acc and 2 in acc))
     assert accepted[:, 0].all() and (accepted.sum(axis=1) > 1).any() and seen_multi > 0
+    assert (accepted.sum(axis=1) < K).any()                    # and something was rejected
 
 
 def test_a_second_parent_rescues_a_node():

@@ -19,7 +19,7 @@ def _free_port():
     return port
 
 
-def _worker(rank, world, port, out):
+def _worker(rank, world, port, out, V=1000):
     sys.path.insert(0, ROOT)
     os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
                       MASTER_PORT=str(port))
@@ -28,19 +28,22 @@ def _worker(rank, world, port, out):
 
     import oracle
     import psd_inputs as gen
-    from paper_2605_15609_b200.vocab_parallel import gather_partials, shard_rows
+    from paper_2605_15609_b200.vocab_parallel import gather_partials, neutral_triple, shard_rows
     dist.init_process_group(backend="gloo", rank=rank, world_size=world)
     rng = np.random.default_rng(0)                      # the same inputs on every rank
-    R, H, V = 9, 64, 1000
+    R, H = 9, 64
     W = gen.bf16_bits(rng.normal(scale=0.2, size=(V, H)).astype(np.float32))
     hid = gen.bf16_bits(rng.normal(size=(R, H)).astype(np.float32))
     v0, v1 = shard_rows(V, world, rank)
-    logits = oracle.logits(hid, W[v0:v1])               # [R, v1 - v0] fp64
-    m = logits.max(axis=1)
-    s = np.exp(logits - m[:, None]).sum(axis=1)
-    a = logits.argmax(axis=1) + v0
-    local = torch.from_numpy(np.stack([m.astype(np.float32).view(np.int32), s.astype(np.float32).view(np.int32),
-                                       a.astype(np.int32)]))
+    if v1 > v0:
+        logits = oracle.logits(hid, W[v0:v1])           # [R, v1 - v0] fp64
+        m = logits.max(axis=1)
+        s = np.exp(logits - m[:, None]).sum(axis=1)
+        a = logits.argmax(axis=1) + v0
+        local = torch.from_numpy(np.stack([m.astype(np.float32).view(np.int32),
+                                           s.astype(np.float32).view(np.int32), a.astype(np.int32)]))
+    else:
+        local = neutral_triple(R)                       # a rank without vocabulary rows still takes part
     allp = gather_partials(local).numpy()               # [world, 3, R]
     ms, ss, aa = allp[:, 0].view(np.float32).astype(np.float64), allp[:, 1].view(np.float32).astype(np.float64), allp[:, 2]
     best = ms.max(axis=0)
@@ -66,6 +69,23 @@ def test_two_ranks_exchange_and_merge():
     (r0, sh0, ok0, e0), (r1, sh1, ok1, e1) = res
     assert sh0 == (0, 512) and sh1 == (512, 1000)
     assert ok0 and ok1 and e0 < 1e-6 and e1 < 1e-6
+
+
+def test_more_ranks_than_ranges_of_sixteen_rows():
+    # V = 20 gives two ranges of the vocabulary; the third rank holds none, contributes the neutral triple
+    # (-inf, 0, INT32_MAX) and must neither stall the all-gather nor change the result
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 3, port, q, 20)) for r in range(3)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [r[1] for r in res] == [(0, 16), (16, 20), (20, 20)]
+    assert all(ok and err < 1e-6 for _, _, ok, err in res)
 
 
 def test_shard_rows_cover_the_vocabulary():
