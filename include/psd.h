@@ -489,8 +489,9 @@ int psd_set_confidence_impl(int impl);
  */
 #define PSD_TUNE_BAND_BYTES 1
 /*   PSD_TUNE_PDL         1 (default): consecutive kernels of a step are launched with programmatic stream
- *                        serialization, so a kernel's set-up overlaps the end of the one before it;
- *                        0: plain stream order */
+ *                        serialization, so a kernel's set-up overlaps the end of the one before it (the
+ *                        fused kernel itself starts early only when the batch is a single row tile);
+ *                        2: the fused kernel starts early at every size; 0: plain stream order */
 #define PSD_TUNE_PDL 2
 /*   PSD_TUNE_TILE_ORDER  0 (default): the library picks the tile order with the smaller estimated DRAM
  *                        traffic; 1: bands of vocabulary tiles (W resident, hidden re-read per band);

@@ -43,7 +43,7 @@ constexpr int kCombineThreads = kCombineRows * kCombineLanes;
 // partial results of its row in lane order.  `sh` is this group's scratch [8][32].
 // Every thread of the group must call this (it synchronises the whole block twice).
 __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, const float* __restrict__ ps,
-                                               const int32_t* __restrict__ pa, int n_split, int n_rows,
+                                               const int32_t* __restrict__ pa, const SplitPlan& plan, int n_rows,
                                                int row0, int row_end, int g, Triple (*sh)[kCombineRows],
                                                int32_t* __restrict__ out_token, float* __restrict__ out_conf,
                                                float* __restrict__ out_lse, const int32_t* __restrict__ pos = nullptr,
@@ -55,6 +55,11 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
     const int row = out_row < row_end ? (pos ? pos[out_row] : out_row) : -1;
     Triple x{-INFINITY, 0.f, INT32_MAX};
     if (row >= 0) {
+        int n_split = plan.uniform;
+        if (n_split <= 0) {
+            const int scored = plan.n_rows_dev ? min(max(*plan.n_rows_dev, 0), plan.n_rows) : plan.n_rows;
+            n_split = carried_splits(plan.G, plan.hb, (scored + kTileRows - 1) / kTileRows, row / kTileRows);
+        }
         // The merge is a dependent chain, the loads are not: fetch a batch of splits first so that their
         // latencies overlap, then merge them in the same order as a plain loop would.
         constexpr int kBatch = 8;

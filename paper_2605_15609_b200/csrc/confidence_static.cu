@@ -55,7 +55,7 @@ extern "C" int psd_confidence_static(const void* hidden_bf16, const void* w_lm_b
     // Nothing in the scratch has to start at zero: the fused kernel writes every (row, split) triple
     // that the combine pass reads, so whatever an earlier call left behind is overwritten first.
     psd::Partials part = psd::carve_partials(scratch, n_rows, V);
-    const int n_split = psd::launch_confidence_tc(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st);
-    if (n_split < 0) return n_split;
-    return psd::launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, nullptr, nullptr, 0, status_dev);
+    psd::SplitPlan plan;
+    if (int rc = psd::launch_confidence(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st, &plan)) return rc;
+    return psd::launch_combine(part, plan, n_rows, out_token, out_conf, out_lse, st, nullptr, nullptr, 0, status_dev);
 }

@@ -6,8 +6,10 @@
 // (M = 128, N = tile width, K = 16, bf16 x bf16 -> fp32) into one of two TMEM accumulators, and
 // four epilogue warps read the finished accumulator straight out of TMEM (one thread = one row) and
 // fold its columns into a per-row (max, sum-exp, argmax) triple.  Logits never reach shared or
-// global memory.  One triple per (row, vocabulary tile) goes to the workspace; the combine kernel
-// merges them.
+// global memory.  Partial triples go to the workspace and the combine pass merges them: with the
+// carried layout (the usual case) every CTA keeps one running triple per row of each row tile it meets
+// in a band of its tile list, in a small table in shared memory, and writes it once at the band's end
+// (a few dozen triples per row, see SplitPlan); otherwise one triple per (row, vocabulary tile).
 //
 // Persistent CTAs (one per SM) walk a static list of tiles; the vocabulary is cut into tiles whose
 // widths are multiples of 16 and differ by at most 16, so that the tile count can be chosen to
@@ -17,11 +19,17 @@
 // Every wait in the kernel is bounded: when a wait runs out the CTA records PSD_ERR_TIMEOUT,
 // raises a CTA-wide abort flag that all roles poll, drains its own asynchronous work with bounded
 // waits, frees its TMEM and returns.
+#include <algorithm>
 #include <atomic>
 #include "tc_common.cuh"
 
 namespace psd {
 namespace {
+
+constexpr int BARRIER_BYTES = 256;
+constexpr int CARRY_BYTES = kCarryEntries * BLOCK_M * 12;   // carried triples of a CTA (24 KB)
+constexpr int SMEM1_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + BARRIER_BYTES + CARRY_BYTES;
+static_assert(SMEM1_BYTES <= 227 * 1024, "shared memory of the single-CTA kernel");
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b_wide,
@@ -40,6 +48,10 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     uint64_t* drain_bar = acc_empty_bar + 2;      // [1] used only when aborting
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+    // carried triples: [kCarryEntries][BLOCK_M] max, then sum-exp, then argmax
+    float* carry_m = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + BARRIER_BYTES);
+    float* carry_s = carry_m + kCarryEntries * BLOCK_M;
+    int32_t* carry_a = reinterpret_cast<int32_t*>(carry_s + kCarryEntries * BLOCK_M);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_blocks = H / BLOCK_K;
@@ -85,7 +97,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         n_rows_act = min(max(*n_rows_dev, 0), n_rows);
         geo.n_mt = (n_rows_act + BLOCK_M - 1) / BLOCK_M;
     }
-    const int n_tiles = geo.n_mt * geo.n_vt;
+    const int n_mt = geo.n_mt;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -98,9 +110,11 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             const uint64_t pol_h = l2_policy_evict_last();
             int q = 0;        // K-slices issued so far
             bool ok = true;
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-                int m_tile, v_tile, v0, ncols;
-                decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+            TileCursor cur;
+            cur.begin(geo, blockIdx.x, gridDim.x, n_mt);
+            for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
+                if (ev != TileCursor::TILE) continue;
+                const int m_tile = cur.m_tile, v_tile = cur.v_tile, v0 = cur.v0, ncols = cur.ncols;
                 const bool wide = v_tile < geo.rem || geo.rem == 0;
                 const CUtensorMap* mb = wide ? &map_b_wide : &map_b_narrow;
                 const uint32_t bytes = A_BYTES + (uint32_t)ncols * BLOCK_K * 2;
@@ -129,13 +143,14 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (lane == 0) {
             int q = 0, it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
-                int m_tile, v_tile, v0, ncols;
-                decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+            TileCursor cur;
+            cur.begin(geo, blockIdx.x, gridDim.x, n_mt);
+            for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
+                if (ev != TileCursor::TILE) continue;
                 const int acc = it & 1;
                 if (!mbar_wait(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t idesc = umma_idesc(ncols);
+                const uint32_t idesc = umma_idesc(cur.ncols);
                 const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
                 for (int kb = 0; kb < k_blocks; ++kb, ++q) {
                     const int s = q % STAGES;
@@ -152,6 +167,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     umma_commit(&empty_bar[s]);       // the slice can be overwritten once these MMAs are done
                 }
                 if (ok) umma_commit(&acc_full_bar[acc]);
+                ++it;
             }
             if (!ok) {
                 // Aborting: make sure no MMA is still writing TMEM before it is freed.
@@ -167,16 +183,47 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const int row_in_tile = quarter * 32 + lane;
         int it = 0;
         bool ok = true;
-        float run_m = -INFINITY, run_s = 0.f;
-        int run_a = 0;
-        for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++it) {
-            int m_tile, v_tile, v0, ncols;
-            decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+        // carried layout: this thread's entries of the table start neutral (no logit seen)
+        auto reset_carry = [&]() {
+#pragma unroll
+            for (int e = 0; e < kCarryEntries; ++e) {
+                carry_m[e * BLOCK_M + row_in_tile] = -INFINITY;
+                carry_s[e * BLOCK_M + row_in_tile] = 0.f;
+                carry_a[e * BLOCK_M + row_in_tile] = 0;
+            }
+        };
+        if (geo.carry) reset_carry();
+        TileCursor cur;
+        cur.begin(geo, blockIdx.x, gridDim.x, n_mt);
+        for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
+            if (ev == TileCursor::BAND_END) {
+                // The band is over for this CTA: write the triples it carried, one per row of every row tile
+                // of its residue class (those it never reached stay neutral), to its slot of those rows.
+                const int entries = cur.end_h / cur.end_gcd;
+                const int slot = (int)blockIdx.x / cur.end_gcd, base = (int)blockIdx.x % cur.end_gcd;
+                for (int e = 0; e < entries; ++e) {
+                    const int row = (cur.end_m0 + base + e * cur.end_gcd) * BLOCK_M + row_in_tile;
+                    if (row < n_rows_act) {
+                        const size_t o = (size_t)slot * n_rows + row;
+                        pm[o] = carry_m[e * BLOCK_M + row_in_tile];
+                        ps[o] = carry_s[e * BLOCK_M + row_in_tile];
+                        pa[o] = carry_a[e * BLOCK_M + row_in_tile];
+                    }
+                }
+                reset_carry();
+                continue;
+            }
+            const int m_tile = cur.m_tile, v_tile = cur.v_tile, v0 = cur.v0, ncols = cur.ncols;
             const int acc = it & 1;
             if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, abort_flag, status_dev)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
-            if (!geo.carry) { run_m = -INFINITY; run_s = 0.f; run_a = 0; }
+            // A CTA meets the tiles of one row tile in ascending vocabulary order, so a carried triple keeps
+            // the lowest index among equal maxima just as per-tile triples do after the merge.
+            const int entry = geo.carry ? ((m_tile - cur.m0) / cur.gcd) * BLOCK_M + row_in_tile : 0;
+            float run_m = -INFINITY, run_s = 0.f;
+            int run_a = 0;
+            if (geo.carry) { run_m = carry_m[entry]; run_s = carry_s[entry]; run_a = carry_a[entry]; }
             const bool ragged = v0 + ncols > V;      // only the last vocabulary tile can reach past V
             for (int c = 0; c < ncols; c += 32) {
                 float x[32];
@@ -193,16 +240,18 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty_bar[acc]);
-            // A CTA's tiles come in ascending vocabulary order, so a carried triple keeps the lowest
-            // index among equal maxima just as the per-tile triples do after the merge.
-            const bool last_of_cta = t + (int)gridDim.x >= n_tiles;
-            const int row = m_tile * BLOCK_M + row_in_tile;
-            if (row < n_rows_act && (!geo.carry || last_of_cta)) {
-                const size_t o = (size_t)(geo.carry ? (int)blockIdx.x : v_tile) * n_rows + row;
-                pm[o] = run_m;
-                ps[o] = run_s;
-                pa[o] = run_a;
+            if (geo.carry) {
+                carry_m[entry] = run_m; carry_s[entry] = run_s; carry_a[entry] = run_a;
+            } else {
+                const int row = m_tile * BLOCK_M + row_in_tile;
+                if (row < n_rows_act) {
+                    const size_t o = (size_t)v_tile * n_rows + row;
+                    pm[o] = run_m;
+                    ps[o] = run_s;
+                    pa[o] = run_a;
+                }
             }
+            ++it;
         }
     }
 
@@ -222,13 +271,13 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
 }  // namespace
 
 int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
-                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st) {
+                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st, SplitPlan* plan) {
     static std::atomic<unsigned long long> smem_set{0};
-    if (!ensure_dynamic_smem(confidence_tc_kernel, SMEM_BYTES, smem_set)) return PSD_ERR_CUDA;
+    if (!ensure_dynamic_smem(confidence_tc_kernel, SMEM1_BYTES, smem_set)) return PSD_ERR_CUDA;
     const int sms = sm_count();
     TileGeometry g = choose_geometry(n_rows, V, sms, max_splits(V), BLOCK_M, 16);
-    g.carry = g.n_mt == 1 ? 1 : 0;
-    choose_order(g, n_rows, H, V, BLOCK_M, band_bytes(), g.carry ? 1 : tile_order());
+    choose_order(g, n_rows, H, V, BLOCK_M, band_bytes(), tile_order());
+    if (g.n_mt == 1) { g.row_bands = 1; g.band = 1; }   // one row tile: ascending vocabulary order either way
     const int wide_rows = (g.rem ? g.base_units + 1 : g.base_units) * 16;
     const int narrow_rows = g.base_units > 0 ? g.base_units * 16 : wide_rows;
     CUtensorMap map_a, map_bw, map_bn;
@@ -237,24 +286,45 @@ int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, 
         return PSD_ERR_CUDA;
     const int n_tiles = g.n_mt * g.n_vt;
     const int grid = n_tiles < sms ? n_tiles : sms;
+    // Carried partials need row bands, and pay only if they leave fewer triples per row than one per
+    // vocabulary tile would (which also keeps them inside the workspace, sized for that).  With the row
+    // count on the device the band heights are not known here: take the worst case, one slot per CTA.
+    int most_splits = grid;
+    if (!n_rows_dev) {
+        most_splits = 0;
+        for (int m0 = 0; m0 < g.n_mt;) {
+            const int h = band_height(grid, g.band, g.n_mt - m0);
+            most_splits = std::max(most_splits, grid / gcd_int(grid, h));
+            m0 += h;
+        }
+    }
+    g.carry = (g.row_bands && most_splits <= g.n_vt) ? 1 : 0;
+    if (g.carry) {
+        plan->uniform = 0;
+        plan->G = grid;
+        plan->hb = g.band;
+        plan->n_rows = n_rows;
+        plan->n_rows_dev = n_rows_dev;
+    } else {
+        *plan = uniform_splits(g.n_vt);
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = SMEM1_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     // Starting before the kernel ahead has drained hides this kernel's set-up, which matters when the
     // whole pass takes under 200 us (one row tile).  With many row tiles an early start was measured
     // to lengthen the pass by 5-8% (8192 rows), so there the kernel keeps plain stream order.
-    attr[0].val.programmaticStreamSerializationAllowed = (pdl_enabled() && g.n_mt == 1) ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = (pdl_enabled() == 2 || (pdl_enabled() && g.n_mt == 1)) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
                                        part.s, part.a, status_dev, n_rows_dev);
     count_launch();
-    if (e != cudaSuccess) return PSD_ERR_CUDA;
-    return g.carry ? grid : g.n_vt;   // number of split slots written per row
+    return e == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }
 
 }  // namespace psd

@@ -324,7 +324,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 }  // namespace
 
 int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
-                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st) {
+                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st, SplitPlan* plan) {
     static std::atomic<unsigned long long> smem_set{0};
     if (!ensure_dynamic_smem(confidence_tc2_kernel, SMEM2_BYTES, smem_set)) return PSD_ERR_CUDA;
     const int pairs_max = sm_count() / 2;
@@ -347,14 +347,15 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     // early start only for one row tile, as in the single-CTA launcher
-    attr[0].val.programmaticStreamSerializationAllowed = (pdl_enabled() && g.n_mt == 1) ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = (pdl_enabled() == 2 || (pdl_enabled() && g.n_mt == 1)) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc2_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
                                        part.s, part.a, status_dev, n_rows_dev);
     count_launch();
     if (e != cudaSuccess) return PSD_ERR_CUDA;
-    return g.carry ? pairs : g.n_vt;   // number of split slots written per row
+    *plan = uniform_splits(g.carry ? pairs : g.n_vt);   // split slots written per row
+    return PSD_OK;
 }
 
 }  // namespace psd

@@ -247,7 +247,8 @@ struct StepTailArgs {
     const float* pm;
     const float* ps;
     const int32_t* pa;
-    int n_split, n_rows, M;
+    SplitPlan plan;
+    int n_rows, M;
     const int32_t* pos;   // NULL, or the column of each row's partials when rows were compacted
     psd_policy_t p;
     int32_t* tokV;
@@ -280,7 +281,7 @@ __global__ void step_tail_kernel(const StepTailArgs a) {
         // threads of a group without a chunk still take part in the barriers inside
         const int r0 = c < n_chunks ? row_begin + c * kCombineRows : row_end;
         if (grp < groups)
-            combine_rows32(a.pm, a.ps, a.pa, a.n_split, a.n_rows, r0, row_end, g, sh[grp], a.tokV, a.confV,
+            combine_rows32(a.pm, a.ps, a.pa, a.plan, a.n_rows, r0, row_end, g, sh[grp], a.tokV, a.confV,
                            nullptr, a.pos, nullptr, 0, a.status_dev);
     }
     __syncthreads();
@@ -331,7 +332,7 @@ int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma,
     return cudaGetLastError() == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }
 
-int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_policy_t p,
+int launch_step_tail(Partials part, SplitPlan plan, int n_rows, int B, int M, psd_policy_t p,
                      int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
                      int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
                      int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st,
@@ -340,7 +341,7 @@ int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_p
     a.pos = pos;
     a.status_dev = status_dev;
     a.pm = part.m; a.ps = part.s; a.pa = part.a;
-    a.n_split = n_split; a.n_rows = n_rows; a.M = M; a.p = p;
+    a.plan = plan; a.n_rows = n_rows; a.M = M; a.p = p;
     a.tokV = tokV; a.confV = confV;
     a.sigma = sigma; a.n_fill = n_fill; a.draft_tokens = draft_tokens; a.draft_mask = draft_mask;
     a.tokens = tokens; a.mask = mask; a.k_star = k_star; a.n_spec = n_spec; a.n_comm = n_comm;
@@ -357,7 +358,7 @@ int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_p
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled();
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, step_tail_kernel, a);

@@ -41,15 +41,22 @@ int pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 long long band_bytes() { return g_band_bytes.load(std::memory_order_relaxed); }
 int tile_order() { return g_tile_order.load(std::memory_order_relaxed); }
 
-int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
-                         int32_t* status_dev, cudaStream_t st, const int32_t* n_rows_dev) {
+int launch_confidence(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
+                      int32_t* status_dev, cudaStream_t st, SplitPlan* plan, const int32_t* n_rows_dev) {
     const int impl = g_conf_impl.load(std::memory_order_relaxed);
+    if (impl == 1) {
+        // the CUDA-core cross-check kernel scores every row of the buffer, whatever the device-side count
+        const int n_split = launch_confidence_simt(hidden, w, n_rows, H, V, part, st);
+        if (n_split < 0) return n_split;
+        *plan = uniform_splits(n_split);
+        return PSD_OK;
+    }
     // Default choice by measurement (V = 126464, H = 4096): at 129..256 rows one CTA pair covers both row
     // tiles and fetches every W tile once (258-265 us against 276-282 us); at 128 rows and below, and
     // from 257 rows up, the single-CTA kernel is faster or equal (see confidence_tc2.cu).
     const bool pairs = confidence_uses_pairs(impl, n_rows);
-    return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st)
-                 : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st);
+    return pairs ? launch_confidence_tc2(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st, plan)
+                 : launch_confidence_tc1(hidden, w, n_rows, H, V, part, status_dev, n_rows_dev, st, plan);
 }
 }  // namespace psd
 
@@ -107,7 +114,7 @@ int psd_set_tuning(int knob, int value) {
             g_compact.store(value);
             return PSD_OK;
         case PSD_TUNE_PDL:
-            if (value != 0 && value != 1) return PSD_ERR_SHAPE;
+            if (value < 0 || value > 2) return PSD_ERR_SHAPE;
             g_pdl.store(value);
             return PSD_OK;
         default:
@@ -151,16 +158,15 @@ int psd_confidence(const void* hidden_bf16, const void* w_lm_bf16, const int32_t
     }
     const bool timed = t_ev_start && t_ev_stop;
     if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
-    int n_split = g_conf_impl.load() == 1
-                      ? launch_confidence_simt(hidden_bf16, w_lm_bf16, n_rows, H, V, part, st)
-                      : launch_confidence_tc(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st);
+    SplitPlan plan;
+    const int rc = launch_confidence(hidden_bf16, w_lm_bf16, n_rows, H, V, part, status_dev, st, &plan);
     if (timed) {
         cudaError_t e = cudaEventRecord(t_ev_stop, st);
         t_ev_start = t_ev_stop = nullptr;
         if (e != cudaSuccess) return PSD_ERR_CUDA;
     }
-    if (n_split < 0) return n_split;
-    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, nullptr, nullptr, 0, status_dev);
+    if (rc < 0) return rc;
+    return launch_combine(part, plan, n_rows, out_token, out_conf, out_lse, st, nullptr, nullptr, 0, status_dev);
 }
 
 int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const int32_t* row_mask,
@@ -182,16 +188,15 @@ int psd_confidence_masked(const void* hidden_bf16, const void* w_lm_bf16, const 
     if (int e = launch_gather_rows(hidden_bf16, cs.row_ids, cs.count, 0, n_rows, H, cs.hidden, st)) return e;
     const bool timed = t_ev_start && t_ev_stop;
     if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
-    int n_split = g_conf_impl.load() == 1
-                      ? launch_confidence_simt(cs.hidden, w_lm_bf16, n_rows, H, V, part, st)
-                      : launch_confidence_tc(cs.hidden, w_lm_bf16, n_rows, H, V, part, status_dev, st, cs.count);
+    SplitPlan plan;
+    const int rc = launch_confidence(cs.hidden, w_lm_bf16, n_rows, H, V, part, status_dev, st, &plan, cs.count);
     if (timed) {
         cudaError_t e = cudaEventRecord(t_ev_stop, st);
         t_ev_start = t_ev_stop = nullptr;
         if (e != cudaSuccess) return PSD_ERR_CUDA;
     }
-    if (n_split < 0) return n_split;
-    return launch_combine(part, n_split, n_rows, out_token, out_conf, out_lse, st, cs.pos, nullptr, 0, status_dev);
+    if (rc < 0) return rc;
+    return launch_combine(part, plan, n_rows, out_token, out_conf, out_lse, st, cs.pos, nullptr, 0, status_dev);
 }
 
 int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, int32_t n_rows, int32_t H,
@@ -206,11 +211,9 @@ int psd_confidence_partial(const void* hidden_bf16, const void* w_shard_bf16, in
     if (workspace_bytes < psd_workspace_bytes(n_rows, H, V_shard)) return PSD_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     Partials part = carve_partials(workspace, n_rows, V_shard);
-    int n_split = g_conf_impl.load() == 1
-                      ? launch_confidence_simt(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, st)
-                      : launch_confidence_tc(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, status_dev, st);
-    if (n_split < 0) return n_split;
-    return launch_combine(part, n_split, n_rows, out_arg, out_sumexp, nullptr, st, nullptr, out_max, v_offset, status_dev);
+    SplitPlan plan;
+    if (int rc = launch_confidence(hidden_bf16, w_shard_bf16, n_rows, H, V_shard, part, status_dev, st, &plan)) return rc;
+    return launch_combine(part, plan, n_rows, out_arg, out_sumexp, nullptr, st, nullptr, out_max, v_offset, status_dev);
 }
 
 int psd_merge_partials(const float* max, const float* sumexp, const int32_t* arg, int32_t n_shards, int32_t n_rows,
@@ -224,7 +227,8 @@ int psd_merge_partials(const float* max, const float* sumexp, const int32_t* arg
     part.m = const_cast<float*>(max);
     part.s = const_cast<float*>(sumexp);
     part.a = const_cast<int32_t*>(arg);
-    return launch_combine(part, n_shards, n_rows, out_token, out_conf, out_lse, reinterpret_cast<cudaStream_t>(cuda_stream));
+    return launch_combine(part, uniform_splits(n_shards), n_rows, out_token, out_conf, out_lse,
+                          reinterpret_cast<cudaStream_t>(cuda_stream));
 }
 
 int psd_select_unmask(const float* conf, const int32_t* tok, const int32_t* node, int32_t n_nodes,
@@ -312,22 +316,21 @@ static int step_impl(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, i
     // merges the split-V partials and runs acceptance, the policy on node k* and the next drafts.
     const bool timed = t_ev_start && t_ev_stop;
     if (timed && cudaEventRecord(t_ev_start, st) != cudaSuccess) return PSD_ERR_CUDA;
-    int n_split = g_conf_impl.load() == 1
-                      ? launch_confidence_simt(hidden, io->w_lm_bf16, n_rows, H, V, part, st)
-                      : launch_confidence_tc(hidden, io->w_lm_bf16, n_rows, H, V, part, status_dev, st, n_rows_dev);
+    SplitPlan plan;
+    const int rc = launch_confidence(hidden, io->w_lm_bf16, n_rows, H, V, part, status_dev, st, &plan, n_rows_dev);
     if (timed) {
         cudaError_t ce = cudaEventRecord(t_ev_stop, st);
         t_ev_start = t_ev_stop = nullptr;
         if (ce != cudaSuccess) return PSD_ERR_CUDA;
     }
-    if (n_split < 0) return n_split;
+    if (rc < 0) return rc;
     if (!g)
-        return launch_step_tail(part, n_split, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
+        return launch_step_tail(part, plan, n_rows, B, M, p, io->tokV, io->confV, io->sigma, io->n_fill,
                                 io->draft_tokens, io->draft_mask, io->tokens, io->mask, io->k_star,
                                 io->n_spec_accepted, io->n_committed, io->sel, io->n_sel, io->sel_pos, st, pos, status_dev);
     // draft graph: the same stages as separate launches (merge, acceptance over the graph, policy on
     // node k*, next drafts of the graph)
-    if (int e = launch_combine(part, n_split, n_rows, io->tokV, io->confV, nullptr, st, pos, nullptr, 0, status_dev)) return e;
+    if (int e = launch_combine(part, plan, n_rows, io->tokV, io->confV, nullptr, st, pos, nullptr, 0, status_dev)) return e;
     if (int e = psd_verify_accept_dag(io->tokV, io->confV, io->sigma, io->draft_tokens, io->draft_mask, B, M, p, g,
                                       io->tokens, io->mask, io->k_star, io->n_spec_accepted, io->n_committed,
                                       nullptr, cuda_stream))

@@ -29,6 +29,53 @@ inline Partials carve_partials(void* workspace, int n_rows, int V) {
     return p;
 }
 
+// ---- How many partial triples each row has -------------------------------------------------------
+// Either the same number for every row (`uniform` > 0), or the carried layout of the single-CTA
+// tensor-core kernel: its tile list is cut into bands of row tiles, G CTAs share the tiles of a band
+// round-robin, and each CTA carries one running triple per row of every row tile it meets in the band
+// and writes it once at the band's end.  With g = gcd(G, band height), CTA c meets the row tiles
+// m = (c mod g) + e*g of the band, and a row tile is met by the G/g CTAs of one residue class, which
+// write to slots c / g: rows of that band have G/g splits.
+constexpr int kTileRows = 128;       // rows per row tile of the tensor-core kernels
+constexpr int kCarryEntries = 16;    // running triples (row tiles) a CTA can carry per band
+
+struct SplitPlan {
+    int uniform;                 // > 0: splits per row, for every row; 0: carried layout (fields below)
+    int G;                       // CTAs that walked the tile list
+    int hb;                      // nominal band height, in row tiles
+    int n_rows;                  // rows (the capacity when n_rows_dev is given)
+    const int32_t* n_rows_dev;   // NULL, or a device word holding how many rows were scored
+};
+inline SplitPlan uniform_splits(int n) { SplitPlan p = {n, 0, 0, 0, nullptr}; return p; }
+
+__host__ __device__ inline int gcd_int(int a, int b) {
+    while (b) { const int t = a % b; a = b; b = t; }
+    return a;
+}
+// Height (row tiles) of the band that begins when `remaining` row tiles are left: at most hb, shrunk
+// until a CTA has at most kCarryEntries row tiles to carry.  Heights up to kCarryEntries always qualify.
+__host__ __device__ inline int band_height(int G, int hb, int remaining) {
+    int h = remaining < hb ? remaining : hb;
+    while (h / gcd_int(G, h) > kCarryEntries) --h;
+    return h;
+}
+// Splits of the rows of row tile m under the carried layout with n_mt row tiles in all.
+__host__ __device__ inline int carried_splits(int G, int hb, int n_mt, int m) {
+    int m0 = 0;
+    if (n_mt >= hb) {
+        // the leading bands all have the height of a full band: jump over them
+        const int h_full = band_height(G, hb, hb);
+        const int k_full = (n_mt - hb) / h_full + 1;
+        if (m < k_full * h_full) return G / gcd_int(G, h_full);
+        m0 = k_full * h_full;
+    }
+    for (;;) {
+        const int h = band_height(G, hb, n_mt - m0);
+        if (m < m0 + h || h <= 0) return G / gcd_int(G, h > 0 ? h : 1);
+        m0 += h;
+    }
+}
+
 void count_launch(int n = 1);
 
 // 1 when kernels are launched with programmatic stream serialization (a kernel's set-up overlaps the
@@ -39,17 +86,18 @@ int pdl_enabled();
 int launch_confidence_simt(const void* hidden, const void* w, int n_rows, int H, int V,
                            Partials part, cudaStream_t st);
 
-// Tensor-core kernels (tcgen05 + TMA).  Each returns the number of splits written, or < 0 (psd_status).
+// Tensor-core kernels (tcgen05 + TMA).  Each returns PSD_OK or < 0 (psd_status) and fills *plan with the
+// layout of the partial triples it wrote.
 // confidence_tc.cu: one CTA per tile of 128 rows; confidence_tc2.cu: a pair of CTAs per tile of 256 rows.
 // n_rows_dev: NULL, or a device word holding how many of the n_rows rows actually hold data (the rest
 // of the buffer is ignored; n_rows stays the capacity and the stride of the partial arrays).
-int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V,
-                          Partials part, int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st);
-int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V,
-                          Partials part, int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st);
-// psd_api.cu: picks the kernel according to psd_set_confidence_impl.
-int launch_confidence_tc(const void* hidden, const void* w, int n_rows, int H, int V,
-                         Partials part, int32_t* status_dev, cudaStream_t st, const int32_t* n_rows_dev = nullptr);
+int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
+                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st, SplitPlan* plan);
+int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
+                          int32_t* status_dev, const int32_t* n_rows_dev, cudaStream_t st, SplitPlan* plan);
+// psd_api.cu: picks the kernel according to psd_set_confidence_impl (the CUDA-core kernel included).
+int launch_confidence(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
+                      int32_t* status_dev, cudaStream_t st, SplitPlan* plan, const int32_t* n_rows_dev = nullptr);
 
 long long band_bytes();   // psd_api.cu: L2 budget for the operand that a band of the tile order keeps resident
 int tile_order();         // psd_api.cu: 0 = choose, 1 = vocabulary bands, 2 = row bands
@@ -86,7 +134,7 @@ inline CompactSpace carve_compact(void* workspace, int n_rows, int H, int V) {
 // combine.cu: merge n_split partial triples per row.
 // pos: NULL, or for every output row the column that holds its partials (-1: the row was not scored
 // and its outputs are left alone).
-int launch_combine(Partials part, int n_split, int n_rows,
+int launch_combine(Partials part, SplitPlan plan, int n_rows,
                    int32_t* out_token, float* out_conf, float* out_lse, cudaStream_t st,
                    const int32_t* pos = nullptr, float* out_max = nullptr, int32_t arg_offset = 0,
                    int32_t* status_dev = nullptr);
@@ -107,7 +155,7 @@ int launch_accept(const int32_t* tokV, const float* confV, const int32_t* sigma,
                   int32_t* accepted, cudaStream_t st);
 
 // policy.cu: the whole tail of a step in one launch (split-V merge, acceptance, policy, next drafts).
-int launch_step_tail(Partials part, int n_split, int n_rows, int B, int M, psd_policy_t p,
+int launch_step_tail(Partials part, SplitPlan plan, int n_rows, int B, int M, psd_policy_t p,
                      int32_t* tokV, float* confV, int32_t* sigma, int32_t* n_fill, int32_t* draft_tokens,
                      int32_t* draft_mask, int32_t* tokens, int32_t* mask, int32_t* k_star, int32_t* n_spec,
                      int32_t* n_comm, int32_t* sel, int32_t* n_sel, int32_t* sel_pos, cudaStream_t st,

@@ -33,9 +33,10 @@ struct TileGeometry {
     int unit;        // columns per unit of tile width: 16, or 32 for CTA pairs (each CTA holds half a tile)
     int base_units;  // every vocabulary tile has base_units or base_units + 1 units
     int rem;         // the first `rem` vocabulary tiles have base_units + 1
-    int carry;       // 1: a CTA keeps one running triple per row across all its tiles (single row tile)
-                     //    and writes it to split slot blockIdx.x; 0: one triple per (row, vocabulary tile)
-    int band;        // tiles per band of the tile order (see decode_tile)
+    int carry;       // 1: carried partials (see SplitPlan): bands of `band` row tiles, each CTA keeps one running
+                     //    triple per row of every row tile it meets in a band and writes it at the band's end;
+                     //    0: one triple per (row, vocabulary tile), tile order as decode_tile says
+    int band;        // tiles per band of the tile order (see decode_tile, TileCursor)
     int row_bands;   // 0: bands of vocabulary tiles, 1: bands of row tiles
 };
 
@@ -195,6 +196,14 @@ __device__ __forceinline__ uint64_t l2_policy_evict_normal() {
     return p;
 }
 
+// First column and width of vocabulary tile v_tile.
+__device__ __forceinline__ void tile_columns(const TileGeometry& g, int v_tile, int& v0, int& ncols) {
+    const int units0 = v_tile < g.rem ? v_tile * (g.base_units + 1)
+                                      : g.rem * (g.base_units + 1) + (v_tile - g.rem) * g.base_units;
+    v0 = units0 * g.unit;
+    ncols = (v_tile < g.rem ? g.base_units + 1 : g.base_units) * g.unit;
+}
+
 // Tile t -> (row tile, first vocabulary column, width).  The tile list is cut into bands so that
 // one operand stays in L2 while the other streams past it once per band; the SMs work on consecutive
 // t at any moment.
@@ -220,11 +229,57 @@ __device__ __forceinline__ void decode_tile(const TileGeometry& g, int t, int& m
         m_tile = r / width;
         v_tile = band * g.band + (r - m_tile * width);
     }
-    const int units0 = v_tile < g.rem ? v_tile * (g.base_units + 1)
-                                      : g.rem * (g.base_units + 1) + (v_tile - g.rem) * g.base_units;
-    v0 = units0 * g.unit;
-    ncols = (v_tile < g.rem ? g.base_units + 1 : g.base_units) * g.unit;
+    tile_columns(g, v_tile, v0, ncols);
 }
+
+// The sequence of tiles of one CTA (or CTA pair) `c` out of `G`, the same in every role of the kernel.
+//   g.carry == 0: tiles c, c + G, c + 2G, .. of the global list, decoded by decode_tile.
+//   g.carry == 1: the row tiles are cut into bands (heights from band_height: g.band, shrunk so that a
+//     CTA meets at most kCarryEntries row tiles per band); inside a band the order is (vocabulary tile,
+//     row tile) with the row tile fastest, so the band of `hidden` stays in L2 while W streams past it
+//     once, and the G CTAs take the band's tiles round-robin starting again from the band's first tile.
+//     After a CTA's last tile of a band (also when it had none) the cursor reports the band's end once:
+//     that is where the epilogue writes its carried triples.
+struct TileCursor {
+    enum { DONE = 0, TILE = 1, BAND_END = 2 };
+    int c, G, n_mt, n_tiles;
+    int t;                    // flat form: next tile
+    int m0, h, gcd, r;        // carried form: first row tile and height of the current band, gcd(G, h), next local tile
+    // outputs of next()
+    int m_tile, v_tile, v0, ncols;
+    int end_m0, end_h, end_gcd;   // the band that just ended (BAND_END)
+
+    __device__ __forceinline__ void begin(const TileGeometry& g, int c_, int G_, int n_mt_) {
+        c = c_; G = G_; n_mt = n_mt_;
+        n_tiles = n_mt * g.n_vt;
+        t = c;
+        m0 = 0; r = c;
+        h = n_mt > 0 ? band_height(G, g.band, n_mt) : 0;
+        gcd = h > 0 ? gcd_int(G, h) : 1;
+    }
+    __device__ __forceinline__ int next(const TileGeometry& g) {
+        if (!g.carry) {
+            if (t >= n_tiles) return DONE;
+            decode_tile(g, t, m_tile, v_tile, v0, ncols);
+            t += G;
+            return TILE;
+        }
+        if (m0 >= n_mt) return DONE;
+        if (r < h * g.n_vt) {
+            v_tile = r / h;
+            m_tile = m0 + (r - v_tile * h);
+            tile_columns(g, v_tile, v0, ncols);
+            r += G;
+            return TILE;
+        }
+        end_m0 = m0; end_h = h; end_gcd = gcd;
+        m0 += h;
+        h = m0 < n_mt ? band_height(G, g.band, n_mt - m0) : 0;
+        gcd = h > 0 ? gcd_int(G, h) : 1;
+        r = c;
+        return BAND_END;
+    }
+};
 
 // Folds 32 logits (columns col0 .. col0+31 of this thread's row) into the running triple.
 // run_m is kept pre-multiplied by log2(e) in run_ml2 so that the exponent is one FMA.

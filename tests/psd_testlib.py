@@ -35,6 +35,26 @@ def weights_cached(name):
     return W, bf16_dev(W)
 
 
+def golden_confidence(name, wl):
+    """The fp64 oracle's confidence outputs for EVERY row of workload `name` (verification batch: token,
+    conf, lse, gap; stage-1 pass: token1, ...), read from tests/golden/full_size_confidence_<name>.npz.
+    That file is written by tests/golden/make_full_size_confidence.py, which calls only the oracle; it is
+    used only if the SHA-256 digests it stores equal those of the input bytes `wl` holds now."""
+    import hashlib
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", f"full_size_confidence_{name}.npz")
+    assert os.path.exists(path), f"{path} is missing: run tests/golden/make_full_size_confidence.py {name}"
+    sha = lambda a: hashlib.sha256(np.ascontiguousarray(a).tobytes()).hexdigest()
+    with np.load(path) as z:
+        g = {k: z[k] for k in z.files}
+    for key, arr in (("sha256_W", wl.W), ("sha256_hidden", wl.hidden_verify), ("sha256_hidden1", wl.hidden_stage1)):
+        assert str(g[key]) == sha(arr), f"{path}: {key} does not match the generated inputs; regenerate the file"
+    assert g["token"].shape[0] == wl.hidden_verify.shape[0] and g["token1"].shape[0] == wl.hidden_stage1.shape[0]
+    for k in ("gap", "gap1"):
+        g[k] = g[k].astype(np.float64)
+    return g
+
+
 def f32(x) -> float:
     return float(np.float32(x))
 
