@@ -443,6 +443,28 @@ def measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseli
     return res
 
 
+def apply_tuning(specs):
+    """--tune KNOB=VALUE pairs -> library settings; returns what was set, for the record."""
+    import paper_2605_15609_b200 as psd
+    knobs = {"band_bytes": psd.PSD_TUNE_BAND_BYTES, "pdl": psd.PSD_TUNE_PDL, "tile_order": psd.PSD_TUNE_TILE_ORDER,
+             "compact_rows": psd.PSD_TUNE_COMPACT_ROWS}
+    done = {}
+    for spec in specs:
+        name, _, value = spec.partition("=")
+        value = int(value)
+        if name == "kernel":
+            rc = psd.psd_set_confidence_impl(value)
+            rc = 0 if rc >= 0 else rc
+        elif name in knobs:
+            rc = psd.psd_set_tuning(knobs[name], value)
+        else:
+            raise SystemExit(f"--tune: unknown knob {name!r}")
+        if rc != 0:
+            raise SystemExit(f"--tune {spec}: {psd.status_string(rc)}")
+        done[name] = value
+    return done
+
+
 def run_ours(args, names):
     import torch
 
@@ -455,6 +477,7 @@ def run_ours(args, names):
     device = torch.device("cuda", info.local_rank)
     replicas.init_process_group(info)
     peaks, peaks_kind = load_peaks()
+    tuning = apply_tuning(args.tune)
 
     results = []
     for i, name in enumerate(names):
@@ -474,6 +497,8 @@ def run_ours(args, names):
                                      "roofline", "cpu_baseline")})
     for r in results[1:]:
         line[r["config"]["workload"]] = r
+    if tuning:
+        line["tuning"] = tuning
     print(json.dumps(line), flush=True)
     return 0
 
@@ -562,6 +587,9 @@ def main():
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="the K-step timed region is repeated until this much device time has passed (at least "
                          "3 times); the line reports the median region and the spread")
+    ap.add_argument("--tune", action="append", default=[], metavar="KNOB=VALUE",
+                    help="set a performance knob of the library before measuring (band_bytes, pdl, tile_order, "
+                         "compact_rows, or kernel for psd_set_confidence_impl); the line records it under \"tuning\"")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loop", default=None, choices=["one_pass", "two_passes"],
                     help="time the whole decoding loop (psd_decode_blocks) instead of one step; an extra "

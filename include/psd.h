@@ -503,6 +503,17 @@ int psd_set_confidence_impl(int impl);
  *                        psd_compact_workspace_bytes, and entries of tokV / confV that belong to
  *                        committed slots are left as they were (no stage reads them) */
 #define PSD_TUNE_COMPACT_ROWS 4
+/*   PSD_TUNE_WAIT_LIMIT  every wait on a barrier inside the tensor-core kernels gives up after this many
+ *                        THOUSANDS of SM clock cycles (default 4 000 000: about 2 s); the kernel then reports
+ *                        PSD_ERR_TIMEOUT through status_dev, lets its own copies and tensor-core work finish
+ *                        (those waits keep the default limit), frees what it holds and returns normally */
+#define PSD_TUNE_WAIT_LIMIT 5
+/*   PSD_TUNE_SELFTEST_STALL  1: self-test of that give-up path.  In every CTA (in the leading CTA of every
+ *                        pair) the loader, after its first K-slice, waits on a barrier that nothing ever
+ *                        arrives on, so the wait runs out after PSD_TUNE_WAIT_LIMIT and the call ends with
+ *                        PSD_ERR_TIMEOUT in status_dev and invalid outputs; nothing faults and the next call
+ *                        (with 0 here) works as usual.  0 (default): off */
+#define PSD_TUNE_SELFTEST_STALL 6
 /* 1 if PSD_TUNE_COMPACT_ROWS makes a batch of n_rows rows take the compacted path, else 0. */
 int psd_compact_rows_enabled(int32_t n_rows);
 int psd_set_tuning(int knob, int value);

@@ -181,6 +181,8 @@ PSD_TUNE_BAND_BYTES = 1
 PSD_TUNE_PDL = 2
 PSD_TUNE_TILE_ORDER = 3
 PSD_TUNE_COMPACT_ROWS = 4
+PSD_TUNE_WAIT_LIMIT = 5
+PSD_TUNE_SELFTEST_STALL = 6
 
 
 def psd_set_tuning(knob: int, value: int) -> int:

@@ -46,7 +46,8 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     uint64_t* acc_full_bar = bars + 2 * STAGES;   // [2] MMA -> epilogue
     uint64_t* acc_empty_bar = acc_full_bar + 2;   // [2] epilogue -> MMA
     uint64_t* drain_bar = acc_empty_bar + 2;      // [1] used only when aborting
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain_bar + 1);
+    uint64_t* never_bar = drain_bar + 1;          // [1] nothing ever arrives on it (self-test of the give-up path)
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(never_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
     // carried triples: [kCarryEntries][BLOCK_M] max, then sum-exp, then argmax
     float* carry_m = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + BARRIER_BYTES);
@@ -66,6 +67,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             mbar_init(&acc_empty_bar[a], 4);   // one arrival per epilogue warp
         }
         mbar_init(drain_bar, 1);
+        mbar_init(never_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -98,6 +100,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         geo.n_mt = (n_rows_act + BLOCK_M - 1) / BLOCK_M;
     }
     const int n_mt = geo.n_mt;
+    const WaitCtx wc = {abort_flag, status_dev, geo.wait_limit, 0u};
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -120,11 +123,13 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const uint32_t bytes = A_BYTES + (uint32_t)ncols * BLOCK_K * 2;
                 for (int kb = 0; kb < k_blocks; ++kb, ++q) {
                     const int s = q % STAGES;
-                    if (!mbar_wait(&empty_bar[s], ((q / STAGES) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
+                    if (!mbar_wait(&empty_bar[s], ((q / STAGES) & 1) ^ 1, wc)) { ok = false; break; }
                     unsigned char* sa = smem + s * STAGE_BYTES;
                     mbar_arrive_expect_tx(&full_bar[s], bytes);
                     tma_load_2d(sa, &map_a, &full_bar[s], kb * BLOCK_K, m_tile * BLOCK_M, pol_h);
                     tma_load_2d(sa + A_BYTES, mb, &full_bar[s], kb * BLOCK_K, v0, pol_w);
+                    // self-test of the give-up path: a wait that nothing will ever satisfy, one slice in flight
+                    if (geo.stall_test && q == 0 && !mbar_wait(never_bar, 0, wc)) { ok = false; ++q; break; }
                 }
             }
             if (!ok) {
@@ -148,13 +153,13 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
                 if (ev != TileCursor::TILE) continue;
                 const int acc = it & 1;
-                if (!mbar_wait(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
+                if (!mbar_wait(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, wc)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t idesc = umma_idesc(cur.ncols);
                 const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
                 for (int kb = 0; kb < k_blocks; ++kb, ++q) {
                     const int s = q % STAGES;
-                    if (!mbar_wait(&full_bar[s], (q / STAGES) & 1, abort_flag, status_dev)) { ok = false; break; }
+                    if (!mbar_wait(&full_bar[s], (q / STAGES) & 1, wc)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
                     const uint64_t da = umma_smem_desc(a_addr);
@@ -215,7 +220,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             }
             const int m_tile = cur.m_tile, v_tile = cur.v_tile, v0 = cur.v0, ncols = cur.ncols;
             const int acc = it & 1;
-            if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, abort_flag, status_dev)) { ok = false; break; }
+            if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, wc)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
             // A CTA meets the tiles of one row tile in ascending vocabulary order, so a carried triple keeps

@@ -38,6 +38,7 @@ constexpr int STAGES2 = PSD_STAGES2;               // depth of the shared-memory
 constexpr int HALF_N = BLOCK_N / 2;                  // widest half tile of W held by one CTA
 constexpr int B2_BYTES = HALF_N * BLOCK_K * 2;       // 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + B2_BYTES;     // 32 KB
+constexpr long long PAIR_DRAIN_CYCLES = 100000000ll;  // about 50 ms: how long an aborting leader watches one slice
 constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -66,17 +67,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
     return ok != 0;
 }
 // Bounded wait on a barrier that threads of the other CTA arrive on.
-__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  int32_t* status_dev) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait_cluster(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            *abort_flag = 1;
-            if (status_dev) atomicCAS(status_dev, 0, (int)PSD_ERR_TIMEOUT);
+        if (*w.abort_flag) return false;
+        if (clock64() - t0 > w.limit) {
+            raise_abort(w);
             return false;
         }
     }
@@ -139,7 +138,8 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     uint64_t* acc_full_bar = bars + 2 * STAGES2;   // [2]
     uint64_t* acc_empty_bar = acc_full_bar + 2;    // [2] used in the leader
     uint64_t* drain_bar = acc_empty_bar + 2;       // [1] used only when aborting
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain_bar + 1);
+    uint64_t* never_bar = drain_bar + 1;           // [1] nothing ever arrives on it (self-test of the give-up path)
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(never_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -158,6 +158,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             mbar_init(&acc_empty_bar[a], 8);   // one arrival per epilogue warp of the pair
         }
         mbar_init(drain_bar, 1);
+        mbar_init(never_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -187,6 +188,9 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         geo.n_mt = (n_rows_act + 2 * BLOCK_M - 1) / (2 * BLOCK_M);
     }
     const int n_tiles = geo.n_mt * geo.n_vt;
+    // a wait that runs out raises the abort flag of BOTH CTAs of the pair, so they give up together
+    const WaitCtx wc = {abort_flag, status_dev, geo.wait_limit,
+                        map_to_cta(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u)};
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (each CTA)
@@ -209,24 +213,30 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 const int col0 = v0 + (int)rank * half;
                 for (int kb = 0; kb < k_blocks; ++kb, ++q) {
                     const int s = q % STAGES2;
-                    if (!mbar_wait(&empty_bar[s], ((q / STAGES2) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
+                    if (!mbar_wait(&empty_bar[s], ((q / STAGES2) & 1) ^ 1, wc)) { ok = false; break; }
+                    // the partner may have given up while this stage was free: issue nothing more then
+                    if (*abort_flag) { ok = false; break; }
                     unsigned char* sa = smem + s * STAGE2_BYTES;
                     if (leader) mbar_arrive_expect_tx(&full_bar[s], bytes_pair);
                     const uint32_t fb = full0 + (uint32_t)s * 8;
                     tma_load_2d_pair(sa, &map_a, fb, kb * BLOCK_K, row0, pol_h);
                     tma_load_2d_pair(sa + A_BYTES, mb, fb, kb * BLOCK_K, col0, pol_w);
+                    // self-test of the give-up path (leading CTA only): a wait that nothing will ever satisfy
+                    if (geo.stall_test && leader && q == 0 && !mbar_wait(never_bar, 0, wc)) { ok = false; ++q; break; }
                 }
             }
             if (!ok) {
                 // Aborting: no copy may still be in flight when the CTA exits.  The leader can watch its
-                // full barriers (bounded); the other CTA's copies report to the leader's barriers, which
-                // it cannot poll, so it lets a fixed interval pass that is far longer than any copy takes.
+                // full barriers (bounded; a slice whose other half the partner never sent runs that wait
+                // out); the other CTA's copies report to the leader's barriers, which it cannot poll, so
+                // it lets a fixed interval pass that is far longer than any copy takes.  Both CTAs stay
+                // resident until the cluster barrier at the end, so a late byte count still finds its barrier.
                 if (leader) {
                     const int first = q > STAGES2 ? q - STAGES2 : 0;
                     for (int i = first; i < q; ++i) {
                         const long long t0 = clock64();
                         while (!mbar_try_wait(&full_bar[i % STAGES2], (i / STAGES2) & 1) &&
-                               clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+                               clock64() - t0 < PAIR_DRAIN_CYCLES) {}
                     }
                 } else {
                     const long long t0 = clock64();
@@ -243,13 +253,13 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 int m_tile, v_tile, v0, ncols;
                 decode_tile(geo, t, m_tile, v_tile, v0, ncols);
                 const int acc = it & 1;
-                if (!mbar_wait_cluster(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, abort_flag, status_dev)) { ok = false; break; }
+                if (!mbar_wait_cluster(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, wc)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t idesc = umma_idesc_pair(ncols);
                 const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
                 for (int kb = 0; kb < k_blocks; ++kb, ++q) {
                     const int s = q % STAGES2;
-                    if (!mbar_wait(&full_bar[s], (q / STAGES2) & 1, abort_flag, status_dev)) { ok = false; break; }
+                    if (!mbar_wait(&full_bar[s], (q / STAGES2) & 1, wc)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(smem + s * STAGE2_BYTES);
                     const uint64_t da = umma_smem_desc(a_addr);
@@ -280,7 +290,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             int m_tile, v_tile, v0, ncols;
             decode_tile(geo, t, m_tile, v_tile, v0, ncols);
             const int acc = it & 1;
-            if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, abort_flag, status_dev)) { ok = false; break; }
+            if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, wc)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
             if (!geo.carry) { run_m = -INFINITY; run_s = 0.f; run_a = 0; }

@@ -12,6 +12,8 @@ std::atomic<int> g_pdl{1};
 std::atomic<int> g_band_bytes{36 << 20};
 std::atomic<int> g_tile_order{0};
 std::atomic<int> g_compact{0};
+std::atomic<int> g_wait_kcycles{4000000};   // thousands of clock cycles: about 2 s
+std::atomic<int> g_stall_test{0};
 thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -40,6 +42,8 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 int pdl_enabled() { return g_pdl.load(std::memory_order_relaxed); }
 long long band_bytes() { return g_band_bytes.load(std::memory_order_relaxed); }
 int tile_order() { return g_tile_order.load(std::memory_order_relaxed); }
+long long wait_limit_cycles() { return 1000ll * g_wait_kcycles.load(std::memory_order_relaxed); }
+int selftest_stall() { return g_stall_test.load(std::memory_order_relaxed); }
 
 int launch_confidence(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
                       int32_t* status_dev, cudaStream_t st, SplitPlan* plan, const int32_t* n_rows_dev) {
@@ -112,6 +116,14 @@ int psd_set_tuning(int knob, int value) {
         case PSD_TUNE_COMPACT_ROWS:
             if (value < 0 || value > 2) return PSD_ERR_SHAPE;
             g_compact.store(value);
+            return PSD_OK;
+        case PSD_TUNE_WAIT_LIMIT:
+            if (value < 1) return PSD_ERR_SHAPE;
+            g_wait_kcycles.store(value);
+            return PSD_OK;
+        case PSD_TUNE_SELFTEST_STALL:
+            if (value != 0 && value != 1) return PSD_ERR_SHAPE;
+            g_stall_test.store(value);
             return PSD_OK;
         case PSD_TUNE_PDL:
             if (value < 0 || value > 2) return PSD_ERR_SHAPE;

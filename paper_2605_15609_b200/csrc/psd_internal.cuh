@@ -99,6 +99,8 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
 int launch_confidence(const void* hidden, const void* w, int n_rows, int H, int V, Partials part,
                       int32_t* status_dev, cudaStream_t st, SplitPlan* plan, const int32_t* n_rows_dev = nullptr);
 
+long long wait_limit_cycles();   // psd_api.cu: PSD_TUNE_WAIT_LIMIT in clock cycles
+int selftest_stall();            // psd_api.cu: PSD_TUNE_SELFTEST_STALL
 long long band_bytes();   // psd_api.cu: L2 budget for the operand that a band of the tile order keeps resident
 int tile_order();         // psd_api.cu: 0 = choose, 1 = vocabulary bands, 2 = row bands
 

@@ -25,7 +25,9 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 2 * BLOCK_N;           // two accumulators
 constexpr int NUM_THREADS = 192;                 // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s at B200 clocks
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s at B200 clocks: limit of the waits that drain a CTA's
+                                                        // own asynchronous work when it gives up, and the default
+                                                        // limit of every other wait (TileGeometry::wait_limit)
 
 struct TileGeometry {
     int n_mt;        // row tiles (of 128 rows for the single-CTA kernel, of 256 rows for CTA pairs)
@@ -38,6 +40,8 @@ struct TileGeometry {
                      //    0: one triple per (row, vocabulary tile), tile order as decode_tile says
     int band;        // tiles per band of the tile order (see decode_tile, TileCursor)
     int row_bands;   // 0: bands of vocabulary tiles, 1: bands of row tiles
+    long long wait_limit;   // clock cycles after which a wait on a barrier gives up (PSD_TUNE_WAIT_LIMIT)
+    int stall_test;         // 1: self-test of the give-up path, see PSD_TUNE_SELFTEST_STALL
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -67,18 +71,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
+// What a wait needs to know to give up: the CTA's abort flag (every role polls it), where to report,
+// how long to wait, and for a CTA pair the partner's abort flag (an address in the cluster's shared
+// window, 0 for none) so that the two CTAs give up together.
+struct WaitCtx {
+    volatile int* abort_flag;
+    int32_t* status_dev;
+    long long limit;
+    uint32_t partner_flag;
+};
+__device__ __forceinline__ void raise_abort(const WaitCtx& w) {
+    *w.abort_flag = 1;
+    if (w.partner_flag)
+        asm volatile("st.relaxed.cluster.shared::cluster.u32 [%0], %1;" ::"r"(w.partner_flag), "r"(1u) : "memory");
+    // a count of non-finite rows left by an earlier call gives way to the error code
+    if (w.status_dev) atomicMin(w.status_dev, (int)PSD_ERR_TIMEOUT);
+}
+
 // Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status_dev) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& w) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            *abort_flag = 1;
-            if (status_dev) atomicCAS(status_dev, 0, (int)PSD_ERR_TIMEOUT);
+        if (*w.abort_flag) return false;
+        if (clock64() - t0 > w.limit) {
+            raise_abort(w);
             return false;
         }
     }
@@ -392,6 +411,8 @@ TileGeometry choose_geometry(int n_rows, int V, int workers, int max_vt, int til
     g.carry = 0;
     g.band = 1;
     g.row_bands = 0;
+    g.wait_limit = wait_limit_cycles();
+    g.stall_test = selftest_stall();
     return g;
 }
 

@@ -121,3 +121,16 @@ def test_block_shape_and_null_errors():
     assert L.psd_step(None, 1, 32, 256, 1024, p, FAKE, 1 << 30, None, None) == psd.PSD_ERR_NULL
     assert L.psd_step_host(None, 1, 32, 256, 1024, p, FAKE, 1 << 30, None, None) == psd.PSD_ERR_NULL
     assert L.psd_set_confidence_impl(7) == psd.PSD_ERR_SHAPE
+    # knobs: bad values and unknown knobs are refused, good ones accepted and put back
+    assert L.psd_set_tuning(psd.PSD_TUNE_WAIT_LIMIT, 0) == psd.PSD_ERR_SHAPE
+    assert L.psd_set_tuning(psd.PSD_TUNE_WAIT_LIMIT, 4_000_000) == psd.PSD_OK
+    assert L.psd_set_tuning(psd.PSD_TUNE_SELFTEST_STALL, 2) == psd.PSD_ERR_SHAPE
+    assert L.psd_set_tuning(psd.PSD_TUNE_SELFTEST_STALL, 0) == psd.PSD_OK
+    assert L.psd_set_tuning(psd.PSD_TUNE_PDL, 3) == psd.PSD_ERR_SHAPE
+    assert L.psd_set_tuning(psd.PSD_TUNE_PDL, 1) == psd.PSD_OK
+    assert L.psd_set_tuning(99, 0) == psd.PSD_ERR_UNSUPPORTED
+    # psd_merge_partials checks alignment before it launches
+    assert L.psd_merge_partials(FAKE + 2, FAKE, FAKE, 2, 8, FAKE, FAKE, None, None) == psd.PSD_ERR_ALIGN
+    assert L.psd_merge_partials(FAKE, FAKE, FAKE, 2, 8, FAKE, FAKE + 1, None, None) == psd.PSD_ERR_ALIGN
+    assert L.psd_confidence_kernel_name(128) == b"confidence_tc_kernel"
+    assert L.psd_confidence_kernel_name(200) == b"confidence_tc2_kernel"
