@@ -392,10 +392,10 @@ def measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseli
         psd.psd_step_host(hb, pg, staging, stream)
     times_e2e = repeated(lambda i: psd.psd_step_host(hb, pg, staging, stream), args.steps)
     e2e_value = rows_all / statistics.median(times_e2e)
-    # bytes actually moved per step: hidden plus the draft state up (one block, padding included), every
-    # output and the status word down (one block)
+    # bytes actually moved per step: hidden plus the one block up (draft state, and the output slots and the
+    # zeroed status word that travel with it), the same block down
     _, off = psd.psd_step_host_block(B, M, D)
-    h2d = R * H * 2 + off[4]
+    h2d = R * H * 2 + off[14] + 4
     d2h = off[14] + 4
 
     if not info.is_main:

@@ -328,8 +328,15 @@ size_t psd_step_host_block(int32_t B, int32_t M, int32_t D, size_t* offsets);
  * Copies hidden and the draft state host->device into `staging`, runs psd_step, copies every
  * output of io back device->host, and waits for the stream.  io holds HOST pointers
  * (w_lm_bf16 excepted).  staging: device, 256-byte aligned, >= psd_step_host_bytes().
- * status_host: NULL, or receives the device status word (PSD_OK or PSD_ERR_TIMEOUT).
+ * status_host: NULL, or receives the device status word (see "The device status word").
  * Synchronous: returns after the outputs are in host memory.
+ * Batches of 2048 rows or more go up in two pieces (blocks are independent: the step on the first
+ * blocks, then on the rest), the second piece's copy running under the first piece's kernels on an
+ * internal stream; the first such call on a device creates that stream and three events, host-side
+ * objects that live until the process exits.  Results are those of psd_step on the same pieces;
+ * confidences can differ from one psd_step over the whole batch in the last bits (another tiling of
+ * the rows), nothing else does.  With the one-block host layout the block's status word is
+ * written by this call before the copy (the block goes up whole, which zeroes the device's word).
  */
 int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
                   void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream);

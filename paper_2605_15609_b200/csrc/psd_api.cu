@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include "psd_internal.cuh"
 
 namespace psd {
@@ -416,6 +417,47 @@ size_t psd_step_host_bytes(int32_t B, int32_t M, int32_t H, int32_t V, int32_t D
     return staging_layout(B, M, H, V, D).total;
 }
 
+// One internal stream and two events per device for psd_step_host's overlapped copies, created on the
+// first call that needs them and kept until the process exits (host-side objects, no device memory).
+namespace {
+struct CopyLane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t begin = nullptr, chunk[2] = {nullptr, nullptr};
+    bool ready = false;
+    std::mutex in_use;   // one call at a time records and waits on the lane's events
+};
+std::mutex g_lane_mu;
+CopyLane g_lanes[64];
+
+CopyLane* copy_lane() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_lane_mu);
+    CopyLane& l = g_lanes[dev];
+    if (!l.ready) {
+        if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        if (cudaEventCreateWithFlags(&l.begin, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&l.chunk[0], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&l.chunk[1], cudaEventDisableTiming) != cudaSuccess)
+            return nullptr;
+        l.ready = true;
+    }
+    return &l;
+}
+
+// The step on blocks [b0, b1) of a batch: every array of io advanced to block b0.
+psd_step_io_t blocks_from(const psd_step_io_t& io, int b0, int M, int D, int H) {
+    psd_step_io_t c = io;
+    const size_t bm = (size_t)b0 * M, bd = (size_t)b0 * D, bdm = (size_t)b0 * D * M;
+    c.hidden_bf16 = reinterpret_cast<const unsigned char*>(io.hidden_bf16) + bdm * H * 2;
+    c.sigma += bm; c.n_fill += bd; c.draft_tokens += bdm; c.draft_mask += bdm;
+    c.tokV += bdm; c.confV += bdm; c.tokens += bm; c.mask += bm;
+    c.k_star += b0; c.n_spec_accepted += b0; c.n_committed += b0;
+    c.sel += bm; c.n_sel += b0; c.sel_pos += bm;
+    return c;
+}
+}  // namespace
+
 int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int32_t V, psd_policy_t p,
                   void* staging, size_t staging_bytes, int32_t* status_host, void* cuda_stream) {
     if (int e = check_step_io(io)) return e;
@@ -434,29 +476,64 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
     bool ok = true;
     // One block: when the caller's arrays sit in host memory exactly as psd_step_host_block lays them
     // out, the draft state goes up in one copy and every output comes back in one.
-    const unsigned char* hb = reinterpret_cast<const unsigned char*>(io->sigma);
+    unsigned char* hb = reinterpret_cast<unsigned char*>(io->sigma);
     auto at = [&](const void* ptr, size_t off) { return reinterpret_cast<const unsigned char*>(ptr) == hb + (off - s.sigma); };
     const bool one_block = at(io->n_fill, s.n_fill) && at(io->draft_tokens, s.draft_tokens) &&
                            at(io->draft_mask, s.draft_mask) && at(io->tokV, s.tokV) && at(io->confV, s.confV) &&
                            at(io->tokens, s.tokens) && at(io->mask, s.mask) && at(io->k_star, s.k_star) &&
                            at(io->n_spec_accepted, s.n_spec) && at(io->n_committed, s.n_comm) && at(io->sel, s.sel) &&
                            at(io->n_sel, s.n_sel) && at(io->sel_pos, s.sel_pos);
-    auto h2d = [&](size_t off, const void* src, size_t bytes) {
-        ok = ok && cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    auto h2d = [&](size_t off, const void* src, size_t bytes, cudaStream_t on) {
+        ok = ok && cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, on) == cudaSuccess;
     };
     auto d2h = [&](void* dst, size_t off, size_t bytes) {
         ok = ok && cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     };
-    h2d(s.hidden, io->hidden_bf16, R * H * 2);
-    if (one_block) {
-        h2d(s.sigma, io->sigma, s.tokV - s.sigma);
-    } else {
-        h2d(s.sigma, io->sigma, BM * 4);
-        h2d(s.n_fill, io->n_fill, (size_t)B * D * 4);
-        h2d(s.draft_tokens, io->draft_tokens, R * 4);
-        h2d(s.draft_mask, io->draft_mask, R * 4);
+
+    // A large batch goes up in two pieces so that the second copy runs under the first piece's kernels:
+    // blocks are independent, so the step on blocks [0, b_cut) and on [b_cut, B) is two psd_step calls.
+    // The first piece is kept small (only its copy is exposed) but not so small that its kernel runs in
+    // the inefficient range: a quarter of the rows, between 512 and 1024 rows, in whole blocks.
+    int b_cut = B;
+    const size_t rows_per_block = (size_t)D * M;
+    if (R >= 2048 && B >= 2) {
+        size_t first_rows = R / 4;
+        if (first_rows < 512) first_rows = 512;
+        if (first_rows > 1024) first_rows = 1024;
+        b_cut = (int)((first_rows + rows_per_block - 1) / rows_per_block);
+        if (b_cut >= B) b_cut = B;
     }
-    ok = ok && cudaMemsetAsync(d + s.status, 0, 4, st) == cudaSuccess;
+    CopyLane* lane = b_cut < B ? copy_lane() : nullptr;
+    if (b_cut < B && !lane) b_cut = B;     // no internal stream: fall back to one piece
+    std::unique_lock<std::mutex> lane_lock;
+    if (lane) lane_lock = std::unique_lock<std::mutex>(lane->in_use);
+
+    // the small arrays first (inputs; in the one-block form the whole block, whose status word the
+    // host zeroes here, so the device word needs no separate clearing)
+    if (one_block) {
+        *reinterpret_cast<int32_t*>(hb + (s.status - s.sigma)) = 0;
+        h2d(s.sigma, io->sigma, s.status + 4 - s.sigma, st);
+    } else {
+        h2d(s.sigma, io->sigma, BM * 4, st);
+        h2d(s.n_fill, io->n_fill, (size_t)B * D * 4, st);
+        h2d(s.draft_tokens, io->draft_tokens, R * 4, st);
+        h2d(s.draft_mask, io->draft_mask, R * 4, st);
+        ok = ok && cudaMemsetAsync(d + s.status, 0, 4, st) == cudaSuccess;
+    }
+    const unsigned char* hid = reinterpret_cast<const unsigned char*>(io->hidden_bf16);
+    const size_t cut_bytes = (size_t)b_cut * rows_per_block * H * 2;
+    if (b_cut == B) {
+        h2d(s.hidden, hid, R * H * 2, st);
+    } else {
+        // the internal stream starts after everything already queued on the caller's stream (an earlier
+        // call may still be reading the staging area), then carries both copies in order
+        ok = ok && cudaEventRecord(lane->begin, st) == cudaSuccess;
+        ok = ok && cudaStreamWaitEvent(lane->stream, lane->begin, 0) == cudaSuccess;
+        h2d(s.hidden, hid, cut_bytes, lane->stream);
+        ok = ok && cudaEventRecord(lane->chunk[0], lane->stream) == cudaSuccess;
+        h2d(s.hidden + cut_bytes, hid + cut_bytes, R * H * 2 - cut_bytes, lane->stream);
+        ok = ok && cudaEventRecord(lane->chunk[1], lane->stream) == cudaSuccess;
+    }
     if (!ok) return PSD_ERR_CUDA;
 
     psd_step_io_t dev;
@@ -476,9 +553,18 @@ int psd_step_host(const psd_step_io_t* io, int32_t B, int32_t M, int32_t H, int3
     dev.sel = reinterpret_cast<int32_t*>(d + s.sel);
     dev.n_sel = reinterpret_cast<int32_t*>(d + s.n_sel);
     dev.sel_pos = reinterpret_cast<int32_t*>(d + s.sel_pos);
-    int e = psd_step(&dev, B, M, H, V, p, d + s.workspace, need - s.workspace,
-                     reinterpret_cast<int32_t*>(d + s.status), cuda_stream);
-    if (e) return e;
+    int32_t* status_dev = reinterpret_cast<int32_t*>(d + s.status);
+    if (b_cut == B) {
+        if (int e = psd_step(&dev, B, M, H, V, p, d + s.workspace, need - s.workspace, status_dev, cuda_stream)) return e;
+    } else {
+        // the second piece reuses the workspace: stream order puts it after the first piece's last kernel
+        if (cudaStreamWaitEvent(st, lane->chunk[0], 0) != cudaSuccess) return PSD_ERR_CUDA;
+        if (int e = psd_step(&dev, b_cut, M, H, V, p, d + s.workspace, need - s.workspace, status_dev, cuda_stream)) return e;
+        if (cudaStreamWaitEvent(st, lane->chunk[1], 0) != cudaSuccess) return PSD_ERR_CUDA;
+        const psd_step_io_t rest = blocks_from(dev, b_cut, M, D, H);
+        if (int e = psd_step(&rest, B - b_cut, M, H, V, p, d + s.workspace, need - s.workspace, status_dev, cuda_stream)) return e;
+        lane_lock.unlock();
+    }
 
     if (one_block) {
         // [sigma .. status]: the status word lands in the caller's block, at the offset the layout gives it

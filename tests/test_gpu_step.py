@@ -165,6 +165,35 @@ def test_psd_step_host_matches_device_step(name, one_block):
         assert np.array_equal(getattr(hb, k).numpy(), want[k]), k
 
 
+@pytest.mark.parametrize("name", ["class_7b", "batched_serving"])
+def test_psd_step_host_in_two_pieces(name):
+    """2048 rows or more (batched_serving) go up in two pieces whose second copy overlaps the first piece's
+    kernels; class_7b (1536 rows) stays in one piece.  Either way: token ids equal to the device-resident
+    step's, confidences equal up to the rounding order of another tiling, and every integer output
+    what the oracle's stages make of the host path's own confidences, bit for bit."""
+    cfg, wl, w_dev = _workload(name)
+    po, pg = policies(cfg)
+    B, M, D = cfg.B, cfg.M, cfg.D
+    pro_g, chain = gpu_prologue(cfg, bf16_dev(wl.hidden_stage1), w_dev, pg)
+    hv_dev = bf16_dev(wl.hidden_verify)
+    want = gpu_step(step_buffers_from(chain, cfg, hv_dev, w_dev), cfg, pg)
+    hb = psd.host_step_buffers(B, M, D, hv_dev.cpu().pin_memory(), w_dev)
+    for k in ("sigma", "n_fill", "draft_tokens", "draft_mask"):
+        getattr(hb, k).copy_(getattr(chain, k))
+    staging = torch.empty(psd.psd_step_host_bytes(B, M, cfg.H, cfg.V, D), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                       # twice: the second call reuses the staging area and the lane
+        for k in ("sigma", "n_fill", "draft_tokens", "draft_mask"):
+            getattr(hb, k).copy_(getattr(chain, k))
+        assert psd.psd_step_host(hb, pg, staging) == 0
+        tokV, confV = hb.tokV.numpy().copy(), hb.confV.numpy().copy()
+        assert np.array_equal(tokV, want["tokV"])
+        assert np.abs(confV - want["confV"]).max() <= 1e-5
+        pro_o = {k: pro_g[k] for k in ("sigma", "n_fill", "draft_tokens", "draft_mask")}
+        out_o = oracle_step(cfg, tokV, confV, pro_o, po)
+        for k in STEP_INT_OUTPUTS:
+            assert np.array_equal(out_o[k], getattr(hb, k).numpy()), k
+
+
 def test_psd_step_can_be_captured_in_a_cuda_graph():
     """The step is two launches with by-value tensor maps and no host synchronisation, so a stream
     capture of it replays to the same outputs as direct calls."""
