@@ -396,13 +396,28 @@ TileGeometry choose_geometry(int n_rows, int V, int workers, int max_vt, int til
     if (vt_max > max_vt) vt_max = max_vt;
     if (vt_max < vt_min) vt_max = vt_min;
     const long long per_tile_cost = 24;   // in columns
+    // Row tiles that share a vocabulary tile in the tile order (the band height, about: the order is
+    // chosen after the geometry); wide tiles come first in the vocabulary, so with several row tiles
+    // only the first rounds of a band pay the wide width.
+    const int h = g.n_mt < 32 ? g.n_mt : 32;
     long long best = -1;
     int best_vt = vt_min;
     for (int vt = vt_min; vt <= vt_max; ++vt) {
-        const long long width = (long long)((units + vt - 1) / vt) * unit;
+        const long long base = units / vt, rem = units % vt;
+        const long long wide = (rem ? base + 1 : base) * unit, narrow = base * unit;
         const long long tiles = (long long)g.n_mt * vt;
         const long long rounds = (tiles + sms - 1) / sms;
-        const long long cost = rounds * (width + per_tile_cost);
+        long long cost;
+        if (g.n_mt == 1) {
+            cost = rounds * (wide + per_tile_cost);
+        } else {
+            // per band of h row tiles: round j starts at vocabulary tile j * sms / h, wide while that is < rem
+            const long long band_rounds = ((long long)h * vt + sms - 1) / sms;
+            long long wide_rounds = (rem * h + sms - 1) / sms;
+            if (wide_rounds > band_rounds) wide_rounds = band_rounds;
+            const long long band_cost = wide_rounds * wide + (band_rounds - wide_rounds) * narrow + band_rounds * per_tile_cost;
+            cost = band_cost * ((g.n_mt + h - 1) / h);
+        }
         if (best < 0 || cost < best) { best = cost; best_vt = vt; }
     }
     g.n_vt = best_vt;
