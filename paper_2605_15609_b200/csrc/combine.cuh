@@ -58,7 +58,7 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
         int n_split = plan.uniform;
         if (n_split <= 0) {
             const int scored = plan.n_rows_dev ? min(max(*plan.n_rows_dev, 0), plan.n_rows) : plan.n_rows;
-            n_split = carried_splits(plan.G, plan.hb, (scored + kTileRows - 1) / kTileRows, row / kTileRows);
+            n_split = carried_splits(plan.G, plan.hb, (scored + plan.tile_rows - 1) / plan.tile_rows, row / plan.tile_rows);
         }
         // The merge is a dependent chain, the loads are not: fetch a batch of splits first so that their
         // latencies overlap, then merge them in the same order as a plain loop would.

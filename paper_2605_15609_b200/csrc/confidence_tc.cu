@@ -308,6 +308,7 @@ int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, 
         plan->uniform = 0;
         plan->G = grid;
         plan->hb = g.band;
+        plan->tile_rows = BLOCK_M;
         plan->n_rows = n_rows;
         plan->n_rows_dev = n_rows_dev;
     } else {

@@ -6,8 +6,9 @@
 // its own HALF of the W tile, and the tensor cores of both SMs read both halves.  Per 128 x 256 block
 // of logits that is 32 KB per K-slice through L2 and shared memory instead of the single-CTA
 // kernel's 48 KB.  Each CTA keeps the accumulator of its 128 rows in its own TMEM and runs the same
-// epilogue as the single-CTA kernel (thread = row, online max / sum-exp / argmax, one triple per
-// (row, vocabulary tile) to the workspace).  Logits never leave the SM.
+// epilogue as the single-CTA kernel (thread = row, online max / sum-exp / argmax, partial triples
+// carried per row tile of a band and written at the band's end, see SplitPlan).  Logits never leave
+// the SM.
 //
 // Measured on B200 at 8192 rows x 126464 x 4096 this version moves a third less data from L2 to the
 // SMs (66 GB against 99 GB per pass) and keeps the tensor pipe as busy (86-88% of cycles), but a
@@ -26,6 +27,7 @@
 // No TMA load is multicast.  Every wait is bounded as in the single-CTA kernel; both CTAs meet at a
 // cluster barrier before they free TMEM and exit, so neither touches the other's shared memory after
 // that CTA has gone.
+#include <algorithm>
 #include "tc_common.cuh"
 
 namespace psd {
@@ -39,7 +41,10 @@ constexpr int HALF_N = BLOCK_N / 2;                  // widest half tile of W he
 constexpr int B2_BYTES = HALF_N * BLOCK_K * 2;       // 16 KB
 constexpr int STAGE2_BYTES = A_BYTES + B2_BYTES;     // 32 KB
 constexpr long long PAIR_DRAIN_CYCLES = 100000000ll;  // about 50 ms: how long an aborting leader watches one slice
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int BARRIER2_BYTES = 256;
+constexpr int CARRY2_BYTES = kCarryEntries * BLOCK_M * 12;   // carried triples of a CTA (24 KB)
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 /* alignment slack */ + BARRIER2_BYTES + CARRY2_BYTES;
+static_assert(SMEM2_BYTES <= 227 * 1024, "shared memory of the CTA-pair kernel");
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -141,6 +146,10 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     uint64_t* never_bar = drain_bar + 1;           // [1] nothing ever arrives on it (self-test of the give-up path)
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(never_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+    // carried triples: [kCarryEntries][BLOCK_M] max, then sum-exp, then argmax
+    float* carry_m = reinterpret_cast<float*>(smem + STAGES2 * STAGE2_BYTES + BARRIER2_BYTES);
+    float* carry_s = carry_m + kCarryEntries * BLOCK_M;
+    int32_t* carry_a = reinterpret_cast<int32_t*>(carry_s + kCarryEntries * BLOCK_M);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -187,7 +196,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         n_rows_act = min(max(*n_rows_dev, 0), n_rows);
         geo.n_mt = (n_rows_act + 2 * BLOCK_M - 1) / (2 * BLOCK_M);
     }
-    const int n_tiles = geo.n_mt * geo.n_vt;
+    const int n_mt = geo.n_mt;
     // a wait that runs out raises the abort flag of BOTH CTAs of the pair, so they give up together
     const WaitCtx wc = {abort_flag, status_dev, geo.wait_limit,
                         map_to_cta(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u)};
@@ -202,9 +211,11 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             const uint32_t full0 = map_to_cta(smem_u32(&full_bar[0]), 0);   // the leader's full[0]
             int q = 0;
             bool ok = true;
-            for (int t = pair_id; t < n_tiles && ok; t += n_pairs) {
-                int m_tile, v_tile, v0, ncols;
-                decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+            TileCursor cur;
+            cur.begin(geo, pair_id, n_pairs, n_mt);
+            for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
+                if (ev != TileCursor::TILE) continue;
+                const int m_tile = cur.m_tile, v_tile = cur.v_tile, v0 = cur.v0, ncols = cur.ncols;
                 const bool wide = v_tile < geo.rem || geo.rem == 0;
                 const CUtensorMap* mb = wide ? &map_b_wide : &map_b_narrow;
                 const int half = ncols >> 1;
@@ -249,13 +260,14 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         if (leader && lane == 0) {
             int q = 0, it = 0;
             bool ok = true;
-            for (int t = pair_id; t < n_tiles && ok; t += n_pairs, ++it) {
-                int m_tile, v_tile, v0, ncols;
-                decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+            TileCursor cur;
+            cur.begin(geo, pair_id, n_pairs, n_mt);
+            for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
+                if (ev != TileCursor::TILE) continue;
                 const int acc = it & 1;
                 if (!mbar_wait_cluster(&acc_empty_bar[acc], ((it >> 1) & 1) ^ 1, wc)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t idesc = umma_idesc_pair(ncols);
+                const uint32_t idesc = umma_idesc_pair(cur.ncols);
                 const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BLOCK_N);
                 for (int kb = 0; kb < k_blocks; ++kb, ++q) {
                     const int s = q % STAGES2;
@@ -270,6 +282,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     umma_commit_pair(&empty_bar[s]);
                 }
                 if (ok) umma_commit_pair(&acc_full_bar[acc]);
+                ++it;
             }
             if (!ok) {
                 umma_commit_pair(drain_bar);   // nothing may still be writing TMEM when it is freed
@@ -284,16 +297,47 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const uint32_t acc_empty0 = map_to_cta(smem_u32(&acc_empty_bar[0]), 0);   // the leader's acc_empty[0]
         int it = 0;
         bool ok = true;
-        float run_m = -INFINITY, run_s = 0.f;
-        int run_a = 0;
-        for (int t = pair_id; t < n_tiles && ok; t += n_pairs, ++it) {
-            int m_tile, v_tile, v0, ncols;
-            decode_tile(geo, t, m_tile, v_tile, v0, ncols);
+        // carried layout: this thread's entries of the table start neutral (no logit seen)
+        auto reset_carry = [&]() {
+#pragma unroll
+            for (int e = 0; e < kCarryEntries; ++e) {
+                carry_m[e * BLOCK_M + row_in_tile] = -INFINITY;
+                carry_s[e * BLOCK_M + row_in_tile] = 0.f;
+                carry_a[e * BLOCK_M + row_in_tile] = 0;
+            }
+        };
+        if (geo.carry) reset_carry();
+        TileCursor cur;
+        cur.begin(geo, pair_id, n_pairs, n_mt);
+        for (int ev; ok && (ev = cur.next(geo)) != TileCursor::DONE;) {
+            if (ev == TileCursor::BAND_END) {
+                // The band is over for this pair: each CTA writes the triples it carried for its half of
+                // every row tile of the pair's residue class, to the pair's slot of those rows.
+                const int entries = cur.end_h / cur.end_gcd;
+                const int slot = pair_id / cur.end_gcd, base = pair_id % cur.end_gcd;
+                for (int e = 0; e < entries; ++e) {
+                    const int row = (cur.end_m0 + base + e * cur.end_gcd) * 256 + (int)rank * BLOCK_M + row_in_tile;
+                    if (row < n_rows_act) {
+                        const size_t o = (size_t)slot * n_rows + row;
+                        pm[o] = carry_m[e * BLOCK_M + row_in_tile];
+                        ps[o] = carry_s[e * BLOCK_M + row_in_tile];
+                        pa[o] = carry_a[e * BLOCK_M + row_in_tile];
+                    }
+                }
+                reset_carry();
+                continue;
+            }
+            const int m_tile = cur.m_tile, v_tile = cur.v_tile, v0 = cur.v0, ncols = cur.ncols;
             const int acc = it & 1;
             if (!mbar_wait(&acc_full_bar[acc], (it >> 1) & 1, wc)) { ok = false; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BLOCK_N);
-            if (!geo.carry) { run_m = -INFINITY; run_s = 0.f; run_a = 0; }
+            // a pair meets the tiles of one row tile in ascending vocabulary order: a carried triple keeps the
+            // lowest index among equal maxima
+            const int entry = geo.carry ? ((m_tile - cur.m0) / cur.gcd) * BLOCK_M + row_in_tile : 0;
+            float run_m = -INFINITY, run_s = 0.f;
+            int run_a = 0;
+            if (geo.carry) { run_m = carry_m[entry]; run_s = carry_s[entry]; run_a = carry_a[entry]; }
             const bool ragged = v0 + ncols > V;
             for (int c = 0; c < ncols; c += 32) {
                 float x[32];
@@ -308,16 +352,18 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty0 + (uint32_t)acc * 8);
-            // One row tile (at most 256 rows): a pair's tiles come in ascending vocabulary order, so each
-            // thread carries one running triple across them and writes it once, to split slot pair_id.
-            const bool last_of_pair = t + n_pairs >= n_tiles;
-            const int row = m_tile * 256 + (int)rank * BLOCK_M + row_in_tile;
-            if (row < n_rows_act && (!geo.carry || last_of_pair)) {
-                const size_t o = (size_t)(geo.carry ? pair_id : v_tile) * n_rows + row;
-                pm[o] = run_m;
-                ps[o] = run_s;
-                pa[o] = run_a;
+            if (geo.carry) {
+                carry_m[entry] = run_m; carry_s[entry] = run_s; carry_a[entry] = run_a;
+            } else {
+                const int row = m_tile * 256 + (int)rank * BLOCK_M + row_in_tile;
+                if (row < n_rows_act) {
+                    const size_t o = (size_t)v_tile * n_rows + row;
+                    pm[o] = run_m;
+                    ps[o] = run_s;
+                    pa[o] = run_a;
+                }
             }
+            ++it;
         }
     }
 
@@ -339,8 +385,8 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     if (!ensure_dynamic_smem(confidence_tc2_kernel, SMEM2_BYTES, smem_set)) return PSD_ERR_CUDA;
     const int pairs_max = sm_count() / 2;
     TileGeometry g = choose_geometry(n_rows, V, pairs_max, max_splits(V), 2 * BLOCK_M, 32);
-    g.carry = g.n_mt == 1 ? 1 : 0;
-    choose_order(g, n_rows, H, V, 2 * BLOCK_M, band_bytes(), g.carry ? 1 : tile_order());
+    choose_order(g, n_rows, H, V, 2 * BLOCK_M, band_bytes(), tile_order());
+    if (g.n_mt == 1) { g.row_bands = 1; g.band = 1; }   // one row tile: ascending vocabulary order either way
     const int wide_half = (g.rem ? g.base_units + 1 : g.base_units) * 16;      // half of unit 32
     const int narrow_half = g.base_units > 0 ? g.base_units * 16 : wide_half;
     CUtensorMap map_a, map_bw, map_bn;
@@ -349,6 +395,27 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
         return PSD_ERR_CUDA;
     const int n_tiles = g.n_mt * g.n_vt;
     const int pairs = n_tiles < pairs_max ? n_tiles : pairs_max;
+    // carried partials under the same conditions as in the single-CTA launcher
+    int most_splits = pairs;
+    if (!n_rows_dev) {
+        most_splits = 0;
+        for (int m0 = 0; m0 < g.n_mt;) {
+            const int h = band_height(pairs, g.band, g.n_mt - m0);
+            most_splits = std::max(most_splits, pairs / gcd_int(pairs, h));
+            m0 += h;
+        }
+    }
+    g.carry = (g.row_bands && most_splits <= g.n_vt) ? 1 : 0;
+    if (g.carry) {
+        plan->uniform = 0;
+        plan->G = pairs;
+        plan->hb = g.band;
+        plan->tile_rows = 2 * BLOCK_M;
+        plan->n_rows = n_rows;
+        plan->n_rows_dev = n_rows_dev;
+    } else {
+        *plan = uniform_splits(g.n_vt);
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -363,9 +430,7 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc2_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
                                        part.s, part.a, status_dev, n_rows_dev);
     count_launch();
-    if (e != cudaSuccess) return PSD_ERR_CUDA;
-    *plan = uniform_splits(g.carry ? pairs : g.n_vt);   // split slots written per row
-    return PSD_OK;
+    return e == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }
 
 }  // namespace psd

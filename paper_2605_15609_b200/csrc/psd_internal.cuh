@@ -36,17 +36,18 @@ inline Partials carve_partials(void* workspace, int n_rows, int V) {
 // and writes it once at the band's end.  With g = gcd(G, band height), CTA c meets the row tiles
 // m = (c mod g) + e*g of the band, and a row tile is met by the G/g CTAs of one residue class, which
 // write to slots c / g: rows of that band have G/g splits.
-constexpr int kTileRows = 128;       // rows per row tile of the tensor-core kernels
+constexpr int kTileRows = 128;       // rows per row tile of the single-CTA tensor-core kernel (TMEM lanes)
 constexpr int kCarryEntries = 16;    // running triples (row tiles) a CTA can carry per band
 
 struct SplitPlan {
     int uniform;                 // > 0: splits per row, for every row; 0: carried layout (fields below)
     int G;                       // CTAs that walked the tile list
     int hb;                      // nominal band height, in row tiles
+    int tile_rows;               // rows per row tile: 128 (single-CTA kernel) or 256 (CTA pairs)
     int n_rows;                  // rows (the capacity when n_rows_dev is given)
     const int32_t* n_rows_dev;   // NULL, or a device word holding how many rows were scored
 };
-inline SplitPlan uniform_splits(int n) { SplitPlan p = {n, 0, 0, 0, nullptr}; return p; }
+inline SplitPlan uniform_splits(int n) { SplitPlan p = {n, 0, 0, kTileRows, 0, nullptr}; return p; }
 
 __host__ __device__ inline int gcd_int(int a, int b) {
     while (b) { const int t = a % b; a = b; b = t; }
