@@ -10,13 +10,11 @@
 // carried per row tile of a band and written at the band's end, see SplitPlan).  Logits never leave
 // the SM.
 //
-// Measured on B200 at 8192 rows x 126464 x 4096 this version moves a third less data from L2 to the
-// SMs (66 GB against 99 GB per pass) and keeps the tensor pipe as busy (86-88% of cycles), but a
-// pass takes 6.9 ms against the single-CTA kernel's 6.3 ms once the board sits at its power cap
-// (lower SM clocks at the same utilisation).  Where it wins is 129..256 rows: one pair covers both row
-// tiles, so every W tile is fetched once and by one pair (258-265 us against 276-282 us for the
-// single-CTA kernel at 192-256 rows), and that range is where the default uses it; elsewhere it is
-// selected with psd_set_confidence_impl(3).  It is held to the same parity tests.
+// Measured on B200 (V = 126464, H = 4096) this version moves a third less data from L2 to the SMs
+// (66 GB against 99 GB per 8192-row pass) and runs within 2% of the single-CTA kernel from 512 to 8192
+// rows once the board sits at its power cap.  Where it wins is 129..256 rows: one pair covers both row
+// tiles, so every W tile is fetched once and by one pair, and that range is where the default uses it;
+// elsewhere it is selected with psd_set_confidence_impl(3).  It is held to the same parity tests.
 //
 // Roles per CTA: warp 0 = TMA producer (own operands), warp 1 = TMEM allocation, and in the leader
 // CTA (cluster rank 0) the MMA issuer for the pair, warps 2-5 = epilogue.  Barriers:
