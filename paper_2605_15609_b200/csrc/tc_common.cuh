@@ -216,7 +216,7 @@ __device__ __forceinline__ uint64_t l2_policy_evict_normal() {
 }
 
 // First column and width of vocabulary tile v_tile.
-__device__ __forceinline__ void tile_columns(const TileGeometry& g, int v_tile, int& v0, int& ncols) {
+__host__ __device__ __forceinline__ void tile_columns(const TileGeometry& g, int v_tile, int& v0, int& ncols) {
     const int units0 = v_tile < g.rem ? v_tile * (g.base_units + 1)
                                       : g.rem * (g.base_units + 1) + (v_tile - g.rem) * g.base_units;
     v0 = units0 * g.unit;
@@ -231,7 +231,7 @@ __device__ __forceinline__ void tile_columns(const TileGeometry& g, int v_tile, 
 //     `hidden` is fetched once per band.
 //   g.row_bands == 1: bands of g.band row tiles.  Inside a band the order is (vocabulary tile, row
 //     tile) with the row tile fastest: the band of `hidden` is resident, W is fetched once per band.
-__device__ __forceinline__ void decode_tile(const TileGeometry& g, int t, int& m_tile, int& v_tile, int& v0,
+__host__ __device__ __forceinline__ void decode_tile(const TileGeometry& g, int t, int& m_tile, int& v_tile, int& v0,
                                             int& ncols) {
     if (g.row_bands) {
         const int per_band = g.band * g.n_vt;
@@ -268,7 +268,7 @@ struct TileCursor {
     int m_tile, v_tile, v0, ncols;
     int end_m0, end_h, end_gcd;   // the band that just ended (BAND_END)
 
-    __device__ __forceinline__ void begin(const TileGeometry& g, int c_, int G_, int n_mt_) {
+    __host__ __device__ __forceinline__ void begin(const TileGeometry& g, int c_, int G_, int n_mt_) {
         c = c_; G = G_; n_mt = n_mt_;
         n_tiles = n_mt * g.n_vt;
         t = c;
@@ -276,7 +276,7 @@ struct TileCursor {
         h = n_mt > 0 ? band_height(G, g.band, n_mt) : 0;
         gcd = h > 0 ? gcd_int(G, h) : 1;
     }
-    __device__ __forceinline__ int next(const TileGeometry& g) {
+    __host__ __device__ __forceinline__ int next(const TileGeometry& g) {
         if (!g.carry) {
             if (t >= n_tiles) return DONE;
             decode_tile(g, t, m_tile, v_tile, v0, ncols);
