@@ -8,7 +8,7 @@
 // not depend on the child: one 64-bit "pass" word per parent, built with warp votes, turns the
 // per-edge check into   (S_k \ S_p) & ~pass[p] == 0.   One warp then walks the nodes in topological
 // order, its lanes trying the accepted parents of a node in parallel.
-#include "psd_internal.cuh"
+#include "policy_common.cuh"
 
 namespace psd {
 namespace {
@@ -20,13 +20,6 @@ struct DagDev {
     int8_t topo[PSD_MAX_DAG_NODES];          // nodes by (number of ranks, index)
     int8_t node_with_rank[PSD_MAX_DAG_NODES]; // some node that speculates rank j, or -1
 };
-
-__device__ __forceinline__ bool ranks_before(float cj, int j, float ci, int i) {
-    bool nj = isnan(cj), ni = isnan(ci);
-    if (nj != ni) return ni;
-    if (nj) return j < i;
-    return cj > ci || (cj == ci && j < i);
-}
 
 __device__ __forceinline__ uint64_t valid_ranks(int m) { return m >= 64 ? ~0ull : ((1ull << m) - 1ull); }
 
@@ -51,8 +44,7 @@ __global__ void build_dag_kernel(const float* __restrict__ conf, const int32_t* 
     const int m = __syncthreads_count(mk);
     int rank = M;
     if (mk) {
-        rank = 0;
-        for (int j = 0; j < M; ++j) rank += (s_flag[j] && ranks_before(s_conf[j], j, c, i)) ? 1 : 0;
+        rank = rank_among(s_conf, s_flag, M, c, i);
     }
     if (in && i >= m) sigma[st + i] = -1;
     if (mk) sigma[st + rank] = i;
@@ -118,10 +110,7 @@ __global__ void accept_dag_kernel(const int32_t* __restrict__ tokV, const float*
                     n_thr += mt && ct > p.tau;
                     rk += mt && ranks_before(ct, t, ci, i);
                 }
-                int n = max(n_thr, p.k_min);
-                if (p.k_max > 0) n = min(n, p.k_max);
-                n = min(n, n_masked);
-                ok = agree && mi && rk < n;
+                ok = agree && mi && rk < policy_count(n_thr, n_masked, p);
             }
         }
         const uint32_t bits = __ballot_sync(0xffffffffu, ok);

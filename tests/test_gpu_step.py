@@ -165,8 +165,8 @@ def test_psd_step_host_matches_device_step(name, one_block):
         assert np.array_equal(getattr(hb, k).numpy(), want[k]), k
 
 
-@pytest.mark.parametrize("name", ["class_7b", "batched_serving"])
-def test_psd_step_host_in_two_pieces(name):
+@pytest.mark.parametrize("name,one_block", [("class_7b", True), ("batched_serving", True), ("batched_serving", False)])
+def test_psd_step_host_in_two_pieces(name, one_block):
     """2048 rows or more (batched_serving) go up in two pieces whose second copy overlaps the first piece's
     kernels; class_7b (1536 rows) stays in one piece.  Either way: token ids equal to the device-resident
     step's, confidences equal up to the rounding order of another tiling, and every integer output
@@ -177,9 +177,9 @@ def test_psd_step_host_in_two_pieces(name):
     pro_g, chain = gpu_prologue(cfg, bf16_dev(wl.hidden_stage1), w_dev, pg)
     hv_dev = bf16_dev(wl.hidden_verify)
     want = gpu_step(step_buffers_from(chain, cfg, hv_dev, w_dev), cfg, pg)
-    hb = psd.host_step_buffers(B, M, D, hv_dev.cpu().pin_memory(), w_dev)
-    for k in ("sigma", "n_fill", "draft_tokens", "draft_mask"):
-        getattr(hb, k).copy_(getattr(chain, k))
+    hv_host = hv_dev.cpu().pin_memory()
+    hb = (psd.host_step_buffers(B, M, D, hv_host, w_dev) if one_block else
+          psd.StepBuffers.allocate(B, M, D, cfg.H, hv_host, w_dev, "cpu", pin=True))
     staging = torch.empty(psd.psd_step_host_bytes(B, M, cfg.H, cfg.V, D), dtype=torch.uint8, device="cuda")
     for _ in range(2):                       # twice: the second call reuses the staging area and the lane
         for k in ("sigma", "n_fill", "draft_tokens", "draft_mask"):
