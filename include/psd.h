@@ -50,14 +50,18 @@ typedef enum psd_status {
                                  unknown accept_mode, or tau is NaN                                 */
     PSD_ERR_CUDA = -6,        /* a CUDA runtime or driver call failed (launch, tensor-map encode)  */
     PSD_ERR_UNSUPPORTED = -7, /* a reserved argument was used                                      */
-    PSD_ERR_TIMEOUT = -8      /* device side only, via status_dev: a bounded wait inside a kernel
+    PSD_ERR_TIMEOUT = -8,     /* device side only, via status_dev: a bounded wait inside a kernel
                                  ran out; the kernel returned early and its outputs are invalid    */
+    PSD_ERR_INTERNAL = -9     /* device side only, via status_dev, and only from the library's debug
+                                 build (compiled with PSD_DEBUG): a bounds or ring-order check inside
+                                 a kernel failed; the offending access was skipped                  */
 } psd_status;
 
 /*
  * The device status word (`status_dev` of the entry points that take one): a device int32 that the
  * CALLER zeroes.  After the call it holds
- *     < 0   a psd_status code detected on the device (PSD_ERR_TIMEOUT); it is never overwritten;
+ *     < 0   a psd_status code detected on the device (PSD_ERR_TIMEOUT; PSD_ERR_INTERNAL from the debug
+ *           build); it is never replaced by a count;
  *     > 0   PSD_ERR_NONFINITE count: the number of scored rows whose logits held a NaN or an infinity,
  *           so that their confidence is NaN (such a row ranks below every number in the policy and
  *           never exceeds tau; nothing faults);

@@ -8,6 +8,7 @@ raises.
 from __future__ import annotations
 
 import ctypes
+import os
 from dataclasses import dataclass
 
 import torch
@@ -18,7 +19,7 @@ _i32, _i64, _f32, _vp, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_float, cty
 
 PSD_OK = 0
 PSD_ERR_NULL, PSD_ERR_SHAPE, PSD_ERR_ALIGN, PSD_ERR_WORKSPACE = -1, -2, -3, -4
-PSD_ERR_POLICY, PSD_ERR_CUDA, PSD_ERR_UNSUPPORTED, PSD_ERR_TIMEOUT = -5, -6, -7, -8
+PSD_ERR_POLICY, PSD_ERR_CUDA, PSD_ERR_UNSUPPORTED, PSD_ERR_TIMEOUT, PSD_ERR_INTERNAL = -5, -6, -7, -8, -9
 PSD_MAX_M, PSD_MAX_DEPTH = 1024, 64
 ACCEPT_AGREE_AND_CONF, ACCEPT_AGREE_ONLY, ACCEPT_AGREE_AND_POLICY = 0, 1, 2
 
@@ -66,7 +67,9 @@ class PsdError(RuntimeError):
 def _load() -> ctypes.CDLL:
     # build() compares the library's time stamp with the sources' and recompiles when a source is newer,
     # so a stale library is never loaded silently
-    lib = ctypes.CDLL(_build.build())
+    # PSD_B200_DEBUG=1 in the environment selects the debug build of the library (device-side bounds and
+    # ring-order checks that report PSD_ERR_INTERNAL through the status word); same entry points
+    lib = ctypes.CDLL(_build.build(debug=DEBUG_BUILD))
     pol = PsdPolicy
     lib.psd_status_string.restype = ctypes.c_char_p
     lib.psd_status_string.argtypes = [ctypes.c_int]
@@ -133,8 +136,9 @@ def _load() -> ctypes.CDLL:
     return lib
 
 
+DEBUG_BUILD = os.environ.get("PSD_B200_DEBUG", "0") not in ("", "0")
 LIB = _load()
-LIB_PATH = _build.LIB
+LIB_PATH = _build.LIB_DEBUG if DEBUG_BUILD else _build.LIB
 
 
 def status_string(code: int) -> str:

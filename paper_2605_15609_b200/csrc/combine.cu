@@ -11,11 +11,11 @@ __global__ void __launch_bounds__(kCombineThreads)
 combine_kernel(const float* __restrict__ pm, const float* __restrict__ ps, const int32_t* __restrict__ pa,
                const SplitPlan plan, int n_rows, int32_t* __restrict__ out_token, float* __restrict__ out_conf,
                float* __restrict__ out_lse, const int32_t* __restrict__ pos, float* __restrict__ out_max,
-               int32_t arg_offset, int32_t* status_dev) {
+               int32_t arg_offset, int32_t* status_dev, size_t part_cap) {
     __shared__ Triple sh[kCombineLanes][kCombineRows];
     asm volatile("griddepcontrol.wait;" ::: "memory");   // the partials come from the kernel launched before
     combine_rows32(pm, ps, pa, plan, n_rows, blockIdx.x * kCombineRows, n_rows, threadIdx.x, sh, out_token,
-                   out_conf, out_lse, pos, out_max, arg_offset, status_dev);
+                   out_conf, out_lse, pos, out_max, arg_offset, status_dev, part_cap);
 }
 
 }  // namespace
@@ -36,7 +36,7 @@ int launch_combine(Partials part, SplitPlan plan, int n_rows, int32_t* out_token
     const float* ps = part.s;
     const int32_t* pa = part.a;
     cudaError_t e = cudaLaunchKernelEx(&cfg, combine_kernel, pm, ps, pa, plan, n_rows, out_token, out_conf, out_lse, pos,
-                                       out_max, arg_offset, status_dev);
+                                       out_max, arg_offset, status_dev, part.cap);
     count_launch();
     return e == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }

@@ -48,7 +48,7 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
                                                int32_t* __restrict__ out_token, float* __restrict__ out_conf,
                                                float* __restrict__ out_lse, const int32_t* __restrict__ pos = nullptr,
                                                float* __restrict__ out_max = nullptr, int32_t arg_offset = 0,
-                                               int32_t* status_dev = nullptr) {
+                                               int32_t* status_dev = nullptr, size_t part_cap = 0) {
     const int tx = g & 31, lane = g >> 5;
     const int out_row = row0 + tx;
     // with compacted rows the partials of output row r sit in column pos[r]; -1 = the row was not scored
@@ -60,6 +60,9 @@ __device__ __forceinline__ void combine_rows32(const float* __restrict__ pm, con
             const int scored = plan.n_rows_dev ? min(max(*plan.n_rows_dev, 0), plan.n_rows) : plan.n_rows;
             n_split = carried_splits(plan.G, plan.hb, (scored + plan.tile_rows - 1) / plan.tile_rows, row / plan.tile_rows);
         }
+        // debug build: the last split this row reads must lie inside the arrays
+        if (!PSD_DEBUG_OK(part_cap == 0 || (n_split >= 1 && (size_t)(n_split - 1) * n_rows + row < part_cap), status_dev))
+            n_split = 0;
         // The merge is a dependent chain, the loads are not: fetch a batch of splits first so that their
         // latencies overlap, then merge them in the same order as a plain loop would.
         constexpr int kBatch = 8;

@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b_wide,
                      const __grid_constant__ CUtensorMap map_b_narrow, TileGeometry geo, int n_rows, int H, int V,
                      float* __restrict__ pm, float* __restrict__ ps, int32_t* __restrict__ pa,
-                     int32_t* status_dev, const int32_t* __restrict__ n_rows_dev) {
+                     int32_t* status_dev, const int32_t* __restrict__ n_rows_dev, size_t part_cap) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment: required by the 128-byte swizzle pattern shared by TMA and the MMA descriptors
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -49,6 +49,9 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     uint64_t* never_bar = drain_bar + 1;          // [1] nothing ever arrives on it (self-test of the give-up path)
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(never_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+#ifdef PSD_DEBUG
+    volatile int* ring_tag = abort_flag + 1;   // [stages] the K-slice number the loader put in each stage
+#endif
     // carried triples: [kCarryEntries][BLOCK_M] max, then sum-exp, then argmax
     float* carry_m = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + BARRIER_BYTES);
     float* carry_s = carry_m + kCarryEntries * BLOCK_M;
@@ -125,6 +128,9 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const int s = q % STAGES;
                     if (!mbar_wait(&empty_bar[s], ((q / STAGES) & 1) ^ 1, wc)) { ok = false; break; }
                     unsigned char* sa = smem + s * STAGE_BYTES;
+#ifdef PSD_DEBUG
+                    ring_tag[s] = q;
+#endif
                     mbar_arrive_expect_tx(&full_bar[s], bytes);
                     tma_load_2d(sa, &map_a, &full_bar[s], kb * BLOCK_K, m_tile * BLOCK_M, pol_h);
                     tma_load_2d(sa + A_BYTES, mb, &full_bar[s], kb * BLOCK_K, v0, pol_w);
@@ -161,6 +167,9 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                     const int s = q % STAGES;
                     if (!mbar_wait(&full_bar[s], (q / STAGES) & 1, wc)) { ok = false; break; }
                     tc_fence_after();
+#ifdef PSD_DEBUG
+                    PSD_DEBUG_OK(ring_tag[s] == q, status_dev);   // the stage holds the slice this MMA expects
+#endif
                     const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
                     const uint64_t da = umma_smem_desc(a_addr);
                     const uint64_t db = umma_smem_desc(a_addr + A_BYTES);
@@ -208,7 +217,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 const int slot = (int)blockIdx.x / cur.end_gcd, base = (int)blockIdx.x % cur.end_gcd;
                 for (int e = 0; e < entries; ++e) {
                     const int row = (cur.end_m0 + base + e * cur.end_gcd) * BLOCK_M + row_in_tile;
-                    if (row < n_rows_act) {
+                    if (row < n_rows_act && PSD_DEBUG_OK((size_t)slot * n_rows + row < part_cap && e < kCarryEntries, status_dev)) {
                         const size_t o = (size_t)slot * n_rows + row;
                         pm[o] = carry_m[e * BLOCK_M + row_in_tile];
                         ps[o] = carry_s[e * BLOCK_M + row_in_tile];
@@ -226,6 +235,8 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
             // A CTA meets the tiles of one row tile in ascending vocabulary order, so a carried triple keeps
             // the lowest index among equal maxima just as per-tile triples do after the merge.
             const int entry = geo.carry ? ((m_tile - cur.m0) / cur.gcd) * BLOCK_M + row_in_tile : 0;
+            if (!PSD_DEBUG_OK(m_tile >= 0 && m_tile < n_mt && v0 >= 0 && v0 < V && ncols > 0 && ncols <= BLOCK_N &&
+                                  entry >= 0 && entry < kCarryEntries * BLOCK_M, status_dev)) { ok = false; break; }
             float run_m = -INFINITY, run_s = 0.f;
             int run_a = 0;
             if (geo.carry) { run_m = carry_m[entry]; run_s = carry_s[entry]; run_a = carry_a[entry]; }
@@ -249,7 +260,7 @@ confidence_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
                 carry_m[entry] = run_m; carry_s[entry] = run_s; carry_a[entry] = run_a;
             } else {
                 const int row = m_tile * BLOCK_M + row_in_tile;
-                if (row < n_rows_act) {
+                if (row < n_rows_act && PSD_DEBUG_OK((size_t)v_tile * n_rows + row < part_cap, status_dev)) {
                     const size_t o = (size_t)v_tile * n_rows + row;
                     pm[o] = run_m;
                     ps[o] = run_s;
@@ -328,7 +339,7 @@ int launch_confidence_tc1(const void* hidden, const void* w, int n_rows, int H, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
-                                       part.s, part.a, status_dev, n_rows_dev);
+                                       part.s, part.a, status_dev, n_rows_dev, part.cap);
     count_launch();
     return e == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }

@@ -129,7 +129,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b_wide,
                       const __grid_constant__ CUtensorMap map_b_narrow, TileGeometry geo, int n_rows, int H, int V,
                       float* __restrict__ pm, float* __restrict__ ps, int32_t* __restrict__ pa,
-                      int32_t* status_dev, const int32_t* __restrict__ n_rows_dev) {
+                      int32_t* status_dev, const int32_t* __restrict__ n_rows_dev, size_t part_cap) {
     extern __shared__ unsigned char smem_raw[];
     // 1024-byte alignment for the 128-byte swizzle; the dynamic shared memory of both CTAs of a cluster
     // starts at the same offset, so the aligned layouts coincide, as cta_group::2 addressing requires.
@@ -144,6 +144,9 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     uint64_t* never_bar = drain_bar + 1;           // [1] nothing ever arrives on it (self-test of the give-up path)
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(never_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+#ifdef PSD_DEBUG
+    volatile int* ring_tag = abort_flag + 1;   // [stages] the K-slice number the loader put in each stage
+#endif
     // carried triples: [kCarryEntries][BLOCK_M] max, then sum-exp, then argmax
     float* carry_m = reinterpret_cast<float*>(smem + STAGES2 * STAGE2_BYTES + BARRIER2_BYTES);
     float* carry_s = carry_m + kCarryEntries * BLOCK_M;
@@ -226,6 +229,9 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     // the partner may have given up while this stage was free: issue nothing more then
                     if (*abort_flag) { ok = false; break; }
                     unsigned char* sa = smem + s * STAGE2_BYTES;
+#ifdef PSD_DEBUG
+                    if (leader) ring_tag[s] = q;
+#endif
                     if (leader) mbar_arrive_expect_tx(&full_bar[s], bytes_pair);
                     const uint32_t fb = full0 + (uint32_t)s * 8;
                     tma_load_2d_pair(sa, &map_a, fb, kb * BLOCK_K, row0, pol_h);
@@ -271,6 +277,9 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const int s = q % STAGES2;
                     if (!mbar_wait(&full_bar[s], (q / STAGES2) & 1, wc)) { ok = false; break; }
                     tc_fence_after();
+#ifdef PSD_DEBUG
+                    PSD_DEBUG_OK(ring_tag[s] == q, status_dev);   // the stage holds the slice this MMA expects
+#endif
                     const uint32_t a_addr = smem_u32(smem + s * STAGE2_BYTES);
                     const uint64_t da = umma_smem_desc(a_addr);
                     const uint64_t db = umma_smem_desc(a_addr + A_BYTES);
@@ -315,7 +324,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 const int slot = pair_id / cur.end_gcd, base = pair_id % cur.end_gcd;
                 for (int e = 0; e < entries; ++e) {
                     const int row = (cur.end_m0 + base + e * cur.end_gcd) * 256 + (int)rank * BLOCK_M + row_in_tile;
-                    if (row < n_rows_act) {
+                    if (row < n_rows_act && PSD_DEBUG_OK((size_t)slot * n_rows + row < part_cap && e < kCarryEntries, status_dev)) {
                         const size_t o = (size_t)slot * n_rows + row;
                         pm[o] = carry_m[e * BLOCK_M + row_in_tile];
                         ps[o] = carry_s[e * BLOCK_M + row_in_tile];
@@ -333,6 +342,8 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             // a pair meets the tiles of one row tile in ascending vocabulary order: a carried triple keeps the
             // lowest index among equal maxima
             const int entry = geo.carry ? ((m_tile - cur.m0) / cur.gcd) * BLOCK_M + row_in_tile : 0;
+            if (!PSD_DEBUG_OK(m_tile >= 0 && m_tile < n_mt && v0 >= 0 && v0 < V && ncols > 0 && ncols <= BLOCK_N &&
+                                  entry >= 0 && entry < kCarryEntries * BLOCK_M, status_dev)) { ok = false; break; }
             float run_m = -INFINITY, run_s = 0.f;
             int run_a = 0;
             if (geo.carry) { run_m = carry_m[entry]; run_s = carry_s[entry]; run_a = carry_a[entry]; }
@@ -354,7 +365,7 @@ confidence_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 carry_m[entry] = run_m; carry_s[entry] = run_s; carry_a[entry] = run_a;
             } else {
                 const int row = m_tile * 256 + (int)rank * BLOCK_M + row_in_tile;
-                if (row < n_rows_act) {
+                if (row < n_rows_act && PSD_DEBUG_OK((size_t)v_tile * n_rows + row < part_cap, status_dev)) {
                     const size_t o = (size_t)v_tile * n_rows + row;
                     pm[o] = run_m;
                     ps[o] = run_s;
@@ -426,7 +437,7 @@ int launch_confidence_tc2(const void* hidden, const void* w, int n_rows, int H, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, confidence_tc2_kernel, map_a, map_bw, map_bn, g, n_rows, H, V, part.m,
-                                       part.s, part.a, status_dev, n_rows_dev);
+                                       part.s, part.a, status_dev, n_rows_dev, part.cap);
     count_launch();
     return e == cudaSuccess ? PSD_OK : PSD_ERR_CUDA;
 }

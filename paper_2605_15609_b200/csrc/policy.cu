@@ -234,6 +234,7 @@ struct StepTailArgs {
     int32_t *sigma, *n_fill, *draft_tokens, *draft_mask;
     int32_t *tokens, *mask, *k_star, *n_spec, *n_comm, *sel, *n_sel, *sel_pos;
     int32_t* status_dev;   // NULL, or the status word that counts non-finite rows
+    size_t part_cap;       // triples each partial array holds (debug build)
 };
 
 __global__ void step_tail_kernel(const StepTailArgs a) {
@@ -260,7 +261,7 @@ __global__ void step_tail_kernel(const StepTailArgs a) {
         const int r0 = c < n_chunks ? row_begin + c * kCombineRows : row_end;
         if (grp < groups)
             combine_rows32(a.pm, a.ps, a.pa, a.plan, a.n_rows, r0, row_end, g, sh[grp], a.tokV, a.confV,
-                           nullptr, a.pos, nullptr, 0, a.status_dev);
+                           nullptr, a.pos, nullptr, 0, a.status_dev, a.part_cap);
     }
     __syncthreads();
 
@@ -318,6 +319,7 @@ int launch_step_tail(Partials part, SplitPlan plan, int n_rows, int B, int M, ps
     StepTailArgs a;
     a.pos = pos;
     a.status_dev = status_dev;
+    a.part_cap = part.cap;
     a.pm = part.m; a.ps = part.s; a.pa = part.a;
     a.plan = plan; a.n_rows = n_rows; a.M = M; a.p = p;
     a.tokV = tokV; a.confV = confV;

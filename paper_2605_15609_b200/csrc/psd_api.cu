@@ -80,6 +80,7 @@ const char* psd_status_string(int code) {
         case PSD_ERR_CUDA: return "a CUDA call failed";
         case PSD_ERR_UNSUPPORTED: return "a reserved argument was used";
         case PSD_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case PSD_ERR_INTERNAL: return "a debug-build check inside a kernel failed";
         default: return "unknown status";
     }
 }
@@ -240,6 +241,7 @@ int psd_merge_partials(const float* max, const float* sumexp, const int32_t* arg
     part.m = const_cast<float*>(max);
     part.s = const_cast<float*>(sumexp);
     part.a = const_cast<int32_t*>(arg);
+    part.cap = (size_t)n_shards * (size_t)n_rows;
     return launch_combine(part, uniform_splits(n_shards), n_rows, out_token, out_conf, out_lse,
                           reinterpret_cast<cudaStream_t>(cuda_stream));
 }

@@ -18,6 +18,7 @@ struct Partials {
     float* m;      // [n_split][n_rows] running max of the split's logits
     float* s;      // [n_split][n_rows] sum of exp(l - m) over the split
     int32_t* a;    // [n_split][n_rows] lowest vocabulary index attaining m
+    size_t cap;    // triples each array holds (checked by the debug build; 0 = not known)
 };
 
 inline Partials carve_partials(void* workspace, int n_rows, int V) {
@@ -26,6 +27,7 @@ inline Partials carve_partials(void* workspace, int n_rows, int V) {
     p.m = reinterpret_cast<float*>(workspace);
     p.s = p.m + n;
     p.a = reinterpret_cast<int32_t*>(p.s + n);
+    p.cap = n;
     return p;
 }
 
@@ -76,6 +78,19 @@ __host__ __device__ inline int carried_splits(int G, int hb, int n_mt, int m) {
         m0 += h;
     }
 }
+
+// Debug build (-DPSD_DEBUG): index and ring-order checks inside the kernels.  A failed check writes
+// PSD_ERR_INTERNAL to the status word (when there is one) and the caller skips the access; nothing
+// traps.  In the normal build the checks compile to nothing.
+#ifdef PSD_DEBUG
+__device__ __forceinline__ bool debug_check(bool ok, int32_t* status_dev) {
+    if (!ok && status_dev) atomicMin(status_dev, (int)PSD_ERR_INTERNAL);
+    return ok;
+}
+#define PSD_DEBUG_OK(cond, status_dev) (::psd::debug_check((cond), (status_dev)))
+#else
+#define PSD_DEBUG_OK(cond, status_dev) (true)
+#endif
 
 void count_launch(int n = 1);
 

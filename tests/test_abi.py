@@ -32,11 +32,19 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, n), n
 
 
+def test_debug_build_exports_the_same_symbols():
+    from paper_2605_15609_b200 import build
+    lib = ctypes.CDLL(build.build(debug=True))
+    for n in _declared_symbols():
+        assert hasattr(lib, n), n
+    assert psd.status_string(psd.PSD_ERR_INTERNAL) == "a debug-build check inside a kernel failed"
+
+
 def test_binding_has_the_same_names():
     for n in _declared_symbols():
         assert hasattr(binding, n) or n in ("psd_status_string",), n
     assert psd.status_string(0) == "ok"
-    for code in range(-8, 1):
+    for code in range(-9, 1):
         assert psd.status_string(code) != "unknown status"
     assert psd.status_string(-99) == "unknown status"
 
