@@ -44,10 +44,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel, from the ncu captures
 # summarised under profiles/, keyed by (workload, kernel): a capture of another kernel does not count.
 NCU_TRAFFIC = {
-    ("single_request", "confidence_tc_kernel"): (1.0406e9, "profiles/confidence_tc_single_request.md"),
-    ("batched_serving", "confidence_tc_kernel"): (2.1497e9, "profiles/confidence_tc_batched_serving.md"),
-    ("single_request_B2", "confidence_tc2_kernel"): (1.0522e9, "profiles/confidence_tc2_256_rows.md"),
-    ("single_request_B8", "confidence_tc_kernel"): (1.0482e9, "profiles/confidence_tc_1024_rows.md"),
+    ("single_request", "confidence_tc_kernel"): (1.0413e9, "profiles/confidence_tc_single_request.md"),
+    ("batched_serving", "confidence_tc_kernel"): (2.1491e9, "profiles/confidence_tc_batched_serving.md"),
+    ("single_request_B2", "confidence_tc2_kernel"): (1.0534e9, "profiles/confidence_tc2_256_rows.md"),
+    ("single_request_B8", "confidence_tc_kernel"): (1.0492e9, "profiles/confidence_tc_1024_rows.md"),
 }
 
 
