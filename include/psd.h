@@ -457,8 +457,10 @@ size_t psd_decode_scratch_bytes(int32_t B, int32_t M);
  *                   (n_sel, k_star, n_spec_accepted, n_committed); the last three are 0 in iterations
  *                   that stopped after Stage 1
  *   stats           host, out
- * The call is synchronous: after every state update the host reads the number of masked slots (a
- * 4-byte copy and a stream synchronisation) to decide whether to go on.  It allocates nothing.
+ * The call is synchronous: after every state update the host waits for the stream and reads the number
+ * of masked slots, which the counting kernel has written straight into a pinned host word, to decide
+ * whether to go on.  It allocates no device memory; the first call of a host thread allocates that one
+ * 64-byte pinned word, which lives until the process exits (if that fails, the count is copied instead).
  */
 int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int32_t B, int32_t M, int32_t H,
                       int32_t V, psd_policy_t p, const psd_dag_t* g, int32_t order, int32_t max_iterations,

@@ -16,9 +16,13 @@ namespace {
 
 // One thread block per sequence block.  n_masked[b] still holds the count from the previous check:
 // a block that had masked slots then has just been through `passes_since` forward passes.
+// The blocks add their counts into counters[0]; the last block to finish (a ticket from counters[1])
+// takes the sum, leaves both counters at zero for the next check, and publishes (sum, seq) as one
+// 8-byte word: to `publish` when the host gave a mapped pinned word, and to counters[2..3] always.
 __global__ void progress_kernel(const int32_t* __restrict__ mask, int M, int passes_since, int iteration,
-                                int32_t* __restrict__ n_masked, int32_t* __restrict__ total,
-                                int32_t* __restrict__ passes, int32_t* __restrict__ done_iteration) {
+                                int32_t* __restrict__ n_masked, int32_t* __restrict__ counters,
+                                int32_t* __restrict__ passes, int32_t* __restrict__ done_iteration,
+                                unsigned long long* publish, uint32_t seq) {
     const int b = blockIdx.x;
     int mine = 0;
     for (int i = threadIdx.x; i < M; i += blockDim.x) mine += mask[(size_t)b * M + i] != 0;
@@ -32,7 +36,18 @@ __global__ void progress_kernel(const int32_t* __restrict__ mask, int M, int pas
         if (before > 0 && passes) passes[b] += passes_since;
         if (before > 0 && s_sum == 0 && done_iteration) done_iteration[b] = iteration;
         n_masked[b] = s_sum;
-        if (s_sum) atomicAdd(total, s_sum);
+        if (s_sum) atomicAdd(&counters[0], s_sum);
+        __threadfence();
+        if (atomicAdd(&counters[1], 1) == (int)gridDim.x - 1) {
+            const int total = atomicExch(&counters[0], 0);
+            counters[1] = 0;
+            const unsigned long long word = ((unsigned long long)seq << 32) | (uint32_t)total;
+            *reinterpret_cast<volatile unsigned long long*>(counters + 2) = word;
+            if (publish) {
+                *reinterpret_cast<volatile unsigned long long*>(publish) = word;
+                __threadfence_system();
+            }
+        }
     }
 }
 
@@ -78,11 +93,39 @@ __global__ void table_body_kernel(const uint4* __restrict__ table, const int32_t
     for (int j = threadIdx.x; j < H / 8; j += blockDim.x) hidden[dst + j] = table[src + j];
 }
 
-int read_total(int32_t* total_dev, cudaStream_t st, int* out) {
-    int32_t h = 0;
-    if (cudaMemcpyAsync(&h, total_dev, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PSD_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return PSD_ERR_CUDA;
-    *out = h;
+// A pinned, mapped 8-byte word per host thread through which the progress kernel hands the host its
+// result without a copy operation (allocated on the thread's first call, kept until the process exits).
+// NULL if the allocation fails: the result is then copied from the device counters instead.
+unsigned long long* host_word() {
+    thread_local unsigned long long* word = nullptr;
+    thread_local bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        if (cudaHostAlloc(&p, 64, cudaHostAllocPortable | cudaHostAllocMapped) == cudaSuccess) {
+            word = reinterpret_cast<unsigned long long*>(p);
+            *word = 0;
+        } else {
+            (void)cudaGetLastError();
+        }
+    }
+    return word;
+}
+
+// Waits for the stream and returns the sum the progress kernel published with sequence number `seq`.
+int read_total(int32_t* counters, unsigned long long* word, uint32_t seq, cudaStream_t st, int* out) {
+    unsigned long long v = 0;
+    if (word) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return PSD_ERR_CUDA;
+        v = *reinterpret_cast<volatile unsigned long long*>(word);
+    }
+    if (!word || (uint32_t)(v >> 32) != seq) {
+        // no mapped word (or the write has not arrived, which a finished stream rules out): copy the device's
+        if (cudaMemcpyAsync(&v, counters + 2, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PSD_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return PSD_ERR_CUDA;
+        if ((uint32_t)(v >> 32) != seq) return PSD_ERR_CUDA;
+    }
+    *out = (int)(uint32_t)v;
     return PSD_OK;
 }
 
@@ -110,8 +153,8 @@ int psd_table_body(void* user, const int32_t* tokens, const int32_t* mask, int32
 
 size_t psd_decode_scratch_bytes(int32_t B, int32_t M) {
     if (B < 1 || M < 1 || M > PSD_MAX_M) return 0;
-    // n_masked[B], total[1], tok1[B*M], conf1[B*M]
-    return ((size_t)B * 4 + 4 + (size_t)B * M * 8 + 255) / 256 * 256;
+    // n_masked[B] (rounded up to a multiple of 8 bytes), counters[4], tok1[B*M], conf1[B*M]
+    return (((size_t)B * 4 + 7) / 8 * 8 + 16 + (size_t)B * M * 8 + 255) / 256 * 256;
 }
 
 int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int32_t B, int32_t M, int32_t H,
@@ -141,8 +184,8 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
     int32_t* n_masked = reinterpret_cast<int32_t*>(scratch);
-    int32_t* total = n_masked + B;
-    int32_t* tok1 = total + 1;
+    int32_t* counters = n_masked + (B + 1) / 2 * 2;   // 8-byte aligned: [sum, tickets, published word (2)]
+    int32_t* tok1 = counters + 4;
     float* conf1 = reinterpret_cast<float*>(tok1 + (size_t)B * M);
     void* hidden = const_cast<void*>(io->hidden_bf16);
     const int threads = M < 256 ? ((M + 31) / 32) * 32 : 256;
@@ -152,14 +195,22 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
     stats->masked_left = 0;
     bool ok = true;
     auto cuda_ok = [&](cudaError_t e) { ok = ok && e == cudaSuccess; };
+    unsigned long long* word = host_word();
+    unsigned long long* word_dev = nullptr;
+    if (word && cudaHostGetDevicePointer(reinterpret_cast<void**>(&word_dev), word, 0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        word = nullptr;
+        word_dev = nullptr;
+    }
+    uint32_t seq = word ? (uint32_t)(*word >> 32) : 0u;   // continues this thread's numbering
     auto progress = [&](int passes_since, int iteration, int* masked_now) -> int {
-        cuda_ok(cudaMemsetAsync(total, 0, 4, st));
-        progress_kernel<<<B, threads, 0, st>>>(io->mask, M, passes_since, iteration, n_masked, total, passes,
-                                               done_iteration);
+        ++seq;
+        progress_kernel<<<B, threads, 0, st>>>(io->mask, M, passes_since, iteration, n_masked, counters, passes,
+                                               done_iteration, word_dev, seq);
         count_launch();
         cuda_ok(cudaGetLastError());
         if (!ok) return PSD_ERR_CUDA;
-        return read_total(total, st, masked_now);
+        return read_total(counters, word, seq, st, masked_now);
     };
     auto record = [&](int iteration, int have_accept) {
         if (!trace) return;
@@ -169,7 +220,7 @@ int psd_decode_blocks(psd_body_fn body, void* user, const psd_step_io_t* io, int
     };
 
     // the blocks' state as the caller left it: count it once, charge no pass
-    cuda_ok(cudaMemsetAsync(n_masked, 0, (size_t)B * 4, st));
+    cuda_ok(cudaMemsetAsync(n_masked, 0, (size_t)((B + 1) / 2 * 2 + 4) * 4, st));   // counts and counters
     if (passes) cuda_ok(cudaMemsetAsync(passes, 0, (size_t)B * 4, st));
     if (done_iteration) cuda_ok(cudaMemsetAsync(done_iteration, 0xFF, (size_t)B * 4, st));
     int masked = 0;
