@@ -133,6 +133,32 @@ def algorithmic_flops(cfg) -> float:
     return 2.0 * cfg.rows * cfg.V * cfg.H
 
 
+def sustained_copy_gbs(device, seconds=0.5):
+    """A STREAM-style copy (b.copy_(a), 512 MiB each way) run back to back for `seconds`: read + write
+    bytes per second under the same sustained conditions as the timed regions.  Context for the HBM-bound
+    figure, printed beside the fraction of the pod file's (burst) copy bandwidth."""
+    import torch
+    n = 256 << 20
+    a = torch.empty(n, dtype=torch.bfloat16, device=device)
+    b = torch.empty(n, dtype=torch.bfloat16, device=device)
+    a.fill_(1.0)
+    for _ in range(3):
+        b.copy_(a)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps, total = 0, 0.0
+    while total < seconds and reps < 100000:
+        e0.record()
+        for _ in range(20):
+            b.copy_(a)
+        e1.record()
+        torch.cuda.synchronize()
+        total += e0.elapsed_time(e1) * 1e-3
+        reps += 20
+    del a, b
+    return 2.0 * n * 2 * reps / total / 1e9
+
+
 def ridge_rows(peaks) -> float:
     return peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
 
@@ -420,6 +446,10 @@ def measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseli
         achieved = algorithmic_bytes(cfg) / kernel_s / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"copy bandwidth, of {peaks_kind}"}
+        # the same kind of copy, sustained for half a second in this process right after the timed regions
+        copy_now = sustained_copy_gbs(device)
+        roof["copy_gbs_sustained_this_run"] = copy_now
+        roof["frac_of_copy_sustained_this_run"] = achieved / copy_now
     traffic = NCU_TRAFFIC.get((cfg.name, kernel_name))
     roof["traffic"] = traffic[0] if traffic else None
     roof["traffic_source"] = (f"ncu capture summarised in {traffic[1]}; not measured by this run" if traffic else
