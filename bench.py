@@ -396,7 +396,9 @@ def measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseli
                 "gpu_launches": launches}
 
     # ---- the same steps again with an event pair around the fused kernel of every step
-    n_k = max(8, min(args.steps * len(times), 512))
+    # (as many steps as the timed regions held, so that the board is in the same sustained state; at most
+    # 4096 event pairs)
+    n_k = max(8, min(args.steps * len(times), 4096))
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
     for a, b in evs:          # torch creates the CUDA event on first record; the library re-records it later
         a.record(stream)
