@@ -361,7 +361,8 @@ def measure_workload(args, cfg, info, device, peaks, peaks_kind, with_cpu_baseli
 
     def spread(times, n):
         return {"ms_per_step_median": 1e3 * statistics.median(times) / n, "ms_per_step_min": 1e3 * min(times) / n,
-                "ms_per_step_max": 1e3 * max(times) / n, "repeats": len(times), "steps_per_repeat": n,
+                "ms_per_step_max": 1e3 * max(times) / n, "ms_per_step_first": 1e3 * times[0] / n,
+                "repeats": len(times), "steps_per_repeat": n,
                 "timed_seconds": sum(times)}
 
     # ---- device-resident steps: the headline value
